@@ -1,0 +1,181 @@
+/*
+ * fgd.h -- C ABI of the B200 (sm_100a) implementation of the Factored Gossip DiLoCo
+ * outer synchronisation round, computed for all K simulated workers on one GPU.
+ *
+ * Data model.  Worker m's flat parameters are row m of a row-major fp32 matrix
+ * [K, ld] (ld >= P, in elements) in DEVICE memory: theta_prev = z_{m,r} (result of the
+ * previous outer step, start of the inner loop), theta_local = y_{m,r,H} (after the H
+ * inner steps), momentum = v_{m,r} (Nesterov outer momentum), theta_new = z_{m,r+1}.
+ * The paper stacks workers as columns X in R^{d x M}; this is the transpose, so
+ * "communication" between workers is a read of another row of the same matrix.
+ *
+ * One round (Sec. 4.1 round equations; Algorithm 1):
+ *     x_m      = Mix1(theta_prev)_m                    non-blocking mix, side stream
+ *     g_m      = theta_prev_m - theta_local_m          = -Delta_m (outer gradient)
+ *     ghat_m   = Mix2(g)_m                             blocking mix
+ *     v'_m     = mu v_m + ghat_m                       Nesterov SGD, App. B
+ *     theta_new_m = x_m - gamma (ghat_m + mu v'_m)
+ *     s_m      = sum_p (theta_new[m][p] - mean_p)^2    consensus distance, Sec. 4.4 / App. D
+ * Mix_W(v)_m = sum_n W[m][n] v_n with W symmetric and doubly stochastic (Sec. 3): ROW
+ * convention, row m of W = the weights worker m applies.
+ *
+ * Conventions for every function.
+ *  - Returns FGD_OK (0) or a negative fgd_status.  Never throws, aborts, exits or prints.
+ *    fgd_last_error() gives a human-readable reason for the last failure on that context.
+ *  - Pointers named theta_*, momentum, g, in, out, x, cd_sumsq are DEVICE pointers on the
+ *    context's device; everything inside fgd_mix_desc and every argument of the host helpers
+ *    (fgd_topo_*, fgd_edge_mask, fgd_effective_weights, fgd_dense_matrix, fgd_cd_finalize) is
+ *    HOST memory.
+ *  - Ownership: the caller owns all tensors.  The library allocates no parameter-sized
+ *    memory and keeps no caller pointer after a call returns; descriptors are consumed
+ *    (copied into the launch) before the call returns.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
+ *    stream): tensors must stay alive until the stream reaches that point.
+ *  - Fast path: base pointers 16-byte aligned and ld % 4 == 0; otherwise an element-wise
+ *    path is used (slower, not an error).
+ *  - Deterministic: the same inputs give bit-identical outputs (no floating-point atomics).
+ *  - fgd_outer_step (with cd_sumsq) and fgd_consensus_distance use the context's small
+ *    partial-sum scratch: two such calls on one context must be ordered on the GPU
+ *    (same stream or an event); all other calls may overlap freely.
+ */
+#ifndef FGD_H_
+#define FGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FGD_MAX_K 64 /* most workers (rows) */
+#define FGD_MAX_D 8  /* most neighbour slots per worker in a sparse mix */
+
+typedef enum {
+  FGD_OK = 0,
+  FGD_ERR_INVALID_ARG = -1, /* NULL pointer, size out of range, malformed descriptor */
+  FGD_ERR_ALIGNMENT = -2,   /* reserved: misalignment is handled by the element-wise path */
+  FGD_ERR_ALIAS = -3,       /* forbidden overlap between tensors */
+  FGD_ERR_UNSUPPORTED = -4, /* valid request this build has no kernel for */
+  FGD_ERR_CUDA = -5,        /* a CUDA runtime call failed (message holds the CUDA error) */
+  FGD_ERR_TIMEOUT = -6      /* reserved for bounded device-side waits */
+} fgd_status;
+
+typedef struct fgd_ctx fgd_ctx; /* opaque; owns O(#CTAs * K) doubles of device scratch */
+
+/* Create a context for [K, ld] matrices with P used columns on CUDA device `device`.
+ * 1 <= K <= FGD_MAX_K, 1 <= P <= ld.  Allocates the partial-sum scratch (about 1 MB). */
+int fgd_create(fgd_ctx** out, int device, int K, int64_t P, int64_t ld);
+int fgd_destroy(fgd_ctx* ctx);
+/* Reason of the last failing call on ctx ("" if none); NULL ctx gives the reason of the
+ * last failing fgd_create / host helper on this thread.  The string is owned by the library. */
+const char* fgd_last_error(const fgd_ctx* ctx);
+const char* fgd_status_string(int status);
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t fgd_launch_count(const fgd_ctx* ctx);
+
+/* ---- mixing operators (Sec. 3 "Gossip-based Mixing"; App. A table of (Mix1, Mix2)) ---- */
+typedef enum {
+  FGD_MIX_IDENTITY = 0, /* W = I ("identity": no mixing) */
+  FGD_MIX_MEAN = 1,     /* W = (1/K) 1 1^T ("global all-reduce"); ignores edge_mask, since the
+                           paper's all-reduce restarts until it succeeds (Sec. 5.2) */
+  FGD_MIX_SPARSE = 2,   /* neighbour list + weights (+ per-round edge mask) */
+  FGD_MIX_DENSE = 3     /* explicit K x K matrix */
+} fgd_mix_kind;
+
+/* What happens to the weights when edge_mask drops an edge (the paper only says a missed
+ * exchange gives weaker mixing; these rules are this library's):
+ *  NONE        dropped edges get weight 0, nothing else changes (rows may sum to < 1);
+ *  SELF_ABSORB surviving edges keep their base weight, both endpoints of a dropped edge add
+ *              its base weight to their self weight;
+ *  METROPOLIS  with d'_m = surviving degree, each surviving edge {m,n} gets
+ *              1/(1+max(d'_m,d'_n)) and the self weight is 1 - (row's edge weights).
+ * The last two keep W symmetric and doubly stochastic. */
+typedef enum { FGD_RENORM_NONE = 0, FGD_RENORM_SELF_ABSORB = 1, FGD_RENORM_METROPOLIS = 2 } fgd_renorm;
+
+typedef struct {
+  int32_t kind;             /* fgd_mix_kind */
+  int32_t K;                /* must equal the context's K */
+  int32_t D;                /* SPARSE: neighbour slots per row, 0..FGD_MAX_D */
+  int32_t renorm;           /* fgd_renorm, SPARSE with edge_mask */
+  const int32_t* nbr;       /* SPARSE: [K*D], neighbour of worker m in slot j, -1 = empty.
+                               No self loops, no duplicates in a row, symmetric (n in row m
+                               iff m in row n). */
+  const float* w;           /* SPARSE: [K*D] base edge weights (ignored by METROPOLIS) */
+  const float* w_self;      /* SPARSE: [K] base self weights */
+  const uint8_t* edge_mask; /* SPARSE: [K*D], 1 = alive, 0 = dropped; NULL = all alive.
+                               Must be symmetric. */
+  const float* W;           /* DENSE: [K*K] row-major, W[m*K+n] = weight worker m gives n */
+} fgd_mix_desc;
+
+/* g = theta_prev - theta_local, the negated outer pseudo-gradient Delta_m = y_{m,r,H} -
+ * y_{m,r,0} (Sec. 4.1; Algorithm 1, the "outer pseudo-gradient" line; the sign is the one
+ * OuterOpt receives).  g: [K, ld], may alias neither input. */
+int fgd_outer_grad(fgd_ctx* ctx, const float* theta_prev, const float* theta_local, float* g,
+                   void* stream);
+
+/* out_m = sum_n W[m][n] in_n (Sec. 3, definition of Mix_W), used for Mix1 or any stand-alone
+ * mix.  in: [K, ld].  out: [K, ld] (out == in allowed: in place), or, when out_is_vector != 0
+ * (kind must be FGD_MIX_MEAN), the single averaged row [P]. */
+int fgd_mix(fgd_ctx* ctx, const fgd_mix_desc* desc, const float* in, float* out,
+            int out_is_vector, void* stream);
+
+/* The fused outer step: outer gradient, Mix2, Nesterov update and (optionally) the consensus
+ * partial sums in ONE pass over HBM (reads theta_local, theta_prev, momentum once, writes
+ * theta_new, momentum once).  Sec. 4.1 last three round equations + App. B update.
+ *   mix2        Mix2 applied to the outer gradient (any kind).
+ *   mix1_fused  if non-NULL, Mix1 is ALSO computed in the kernel from theta_prev (kind
+ *               IDENTITY, MEAN or SPARSE) and `x` must be NULL; if NULL, `x` holds the Mix1
+ *               result computed earlier (e.g. by fgd_mix on a side stream): [P] when
+ *               x_is_vector != 0 (the global average), else [K, ld].
+ *   momentum    [K, ld], updated in place.
+ *   theta_new   [K, ld]; may be exactly theta_prev (in place).  No other overlap allowed.
+ *   lr, mu      outer learning rate gamma and momentum mu (used as fp32 in the kernel).
+ *   cd_sumsq    NULL, or device [K] doubles receiving s_m of theta_new (see
+ *               fgd_consensus_distance). */
+int fgd_outer_step(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused,
+                   const float* x, int x_is_vector, const float* theta_local,
+                   const float* theta_prev, float* momentum, float* theta_new, double lr,
+                   double mu, double* cd_sumsq, void* stream);
+
+/* s_m = sum_p (theta[m][p] - (1/K) sum_n theta[n][p])^2 into device cd_sumsq[K] (doubles).
+ * The paper gives two L2 consensus distances, both functions of s: the mean of the
+ * un-squared norms (Sec. 4.4) and the mean of the squared norms (App. D); see
+ * fgd_cd_finalize. */
+int fgd_consensus_distance(fgd_ctx* ctx, const float* theta, double* cd_sumsq, void* stream);
+
+/* ---------------------------- host helpers (pure CPU) ---------------------------------- */
+/* Topologies.  Each writes nbr[K*D], w[K*D], w_self[K] for the D it documents and returns D
+ * (>= 0) or a negative status.  Weights are Metropolis weights of the unmasked graph.
+ *  ring:            D = 2, slots (m-1) mod K, (m+1) mod K; K == 2 uses slot 0 only; 1/3 each.
+ *  onepeer_xor:     D = 1, partner m XOR 2^(round mod log2 K), weight 1/2; K a power of two.
+ *  hypercube:       D = log2 K, slot j = m XOR 2^j, weights 1/(1 + log2 K); K a power of two.
+ *  random_matching: D = 1, one random perfect matching per (seed, round, mix_id), each pair
+ *                   averages (the paper's "pairwise gossip", Sec. 3); odd K leaves one idle. */
+int fgd_topo_ring(int K, int32_t* nbr, float* w, float* w_self);
+int fgd_topo_onepeer_xor(int K, int64_t round, int32_t* nbr, float* w, float* w_self);
+int fgd_topo_hypercube(int K, int32_t* nbr, float* w, float* w_self);
+int fgd_topo_random_matching(int K, uint64_t seed, int64_t round, int mix_id, int32_t* nbr,
+                             float* w, float* w_self);
+/* Transient link failures (Sec. 1, Sec. 5.2): every undirected edge is dropped independently
+ * with probability p_fail in round `round`; mix_id (1 = Mix1, 2 = Mix2) gives the two
+ * transfers of a round independent draws.  Counter-based and order independent: edge {a,b}
+ * is dropped iff the top 32 bits of H(seed, round, mix_id, min, max) are below
+ * floor(p_fail * 2^32).  mask_out[K*D]: 1 alive, 0 dropped or empty slot. */
+int fgd_edge_mask(uint64_t seed, int64_t round, int mix_id, double p_fail, int K, int D,
+                  const int32_t* nbr, uint8_t* mask_out);
+/* The 64-bit hash behind fgd_edge_mask and fgd_topo_random_matching (exposed for tests). */
+uint64_t fgd_hash64(uint64_t seed, uint64_t round, uint64_t tag, uint64_t a, uint64_t b);
+/* Effective weights of a SPARSE descriptor after mask + renormalisation:
+ * w_eff[K*D], w_self_eff[K] (doubles).  Also validates the descriptor. */
+int fgd_effective_weights(const fgd_mix_desc* desc, double* w_eff, double* w_self_eff);
+/* Dense K x K row-convention matrix of any descriptor (doubles, row-major). */
+int fgd_dense_matrix(const fgd_mix_desc* desc, double* W_out);
+/* From s[K] (host doubles): *cd_mean_norm = (1/K) sum sqrt(s_m)  (Sec. 4.4),
+ *                           *cd_mean_sq   = (1/K) sum s_m         (App. D). */
+int fgd_cd_finalize(const double* sumsq_host, int K, double* cd_mean_norm, double* cd_mean_sq);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FGD_H_ */

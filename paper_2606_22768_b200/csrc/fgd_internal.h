@@ -1,0 +1,54 @@
+// Internal declarations shared by the host helpers and the CUDA launch code.
+#ifndef FGD_INTERNAL_H_
+#define FGD_INTERNAL_H_
+
+#include <cstdarg>
+#include <cstddef>
+#include <cstdint>
+
+#include "fgd.h"
+
+namespace fgd {
+
+extern thread_local char g_thread_error[256];
+void set_thread_error(const char* fmt, ...);
+uint64_t hash64(uint64_t seed, uint64_t round, uint64_t tag, uint64_t a, uint64_t b);
+int validate_desc(const fgd_mix_desc* d, int K, char* msg, size_t msg_len);
+void effective_weights(const fgd_mix_desc* d, double* w_eff, double* ws_eff);
+
+// ---- what a kernel receives about a mix, passed BY VALUE as a kernel parameter (it lands
+// in the constant bank, so the warp-uniform reads below are broadcast constant loads).
+enum : int { KMIX_MEAN = 1, KMIX_GATHER = 2 };  // identity is a gather with D = 0, w_self = 1
+
+struct GatherMix {
+  int kind;                            // KMIX_MEAN or KMIX_GATHER
+  int D;                               // used neighbour slots
+  int nbr[FGD_MAX_K * FGD_MAX_D];      // row stride FGD_MAX_D; empty slots point at the row itself
+  float w[FGD_MAX_K * FGD_MAX_D];      // effective weights (0 for dropped / empty slots)
+  float w_self[FGD_MAX_K];             // effective self weights
+};
+
+struct DenseMix {
+  float Wt[FGD_MAX_K * FGD_MAX_K];     // TRANSPOSED, packed with stride K: Wt[n*K+m] = W[m][n]
+};
+
+enum : int { XSRC_VECTOR = 0, XSRC_MATRIX = 1, XSRC_FUSED = 2 };
+
+struct StepArgs {
+  const float* theta_local;
+  const float* theta_prev;
+  float* momentum;
+  float* theta_new;
+  const float* x;       // XSRC_VECTOR: [P]; XSRC_MATRIX: [K, ld]; XSRC_FUSED: unused
+  double* partials;     // [gridDim.x][K] consensus partial sums, or nullptr
+  int64_t P;
+  int64_t ld;
+  int K;
+  int xsrc;
+  int stage_tp;         // 1 when Mix1 is a fused gather (theta_prev columns staged in smem)
+  float lr;
+  float mu;
+};
+
+}  // namespace fgd
+#endif

@@ -1,0 +1,79 @@
+"""Sequencing of one outer round on CUDA streams (Algorithm 1's launch / wait structure).
+
+The paper launches Mix1 asynchronously at the top of a round, runs the H inner steps, then
+blocks on Mix2, waits for Mix1 and applies the outer optimizer.  On one GPU with K workers as
+rows that becomes:
+
+    side stream : Mix1(theta_prev) -> x            (starts once theta_prev is final)
+    main stream : inner steps (whatever produces theta_local)
+    main stream : wait(Mix1) -> fused outer step (outer grad + Mix2 + Nesterov [+ consensus])
+
+This module only orders C-ABI calls with events; all arithmetic is in the library's kernels.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import (FGD_MIX_IDENTITY, FGD_MIX_MEAN, Context, MixDesc, fgd_consensus_distance, fgd_mix,
+               fgd_outer_step)
+
+
+class OuterRound:
+    """Holds the context, the side stream and the Mix1 result buffers for fixed (K, P, ld)."""
+
+    def __init__(self, K: int, P: int, ld: Optional[int] = None, device: int = 0):
+        self.ctx = Context(K, P, ld, device)
+        self.K, self.P, self.ld = self.ctx.K, self.ctx.P, self.ctx.ld
+        self.device = torch.device("cuda", device)
+        self.side = torch.cuda.Stream(device=self.device)
+        self.cd_sumsq = torch.zeros(K, dtype=torch.float64, device=self.device)
+        self._x_vec = None
+        self._x_mat = None
+        self._pending = None  # (event, x tensor, x_is_vector)
+
+    # ---- Mix1: non-blocking, on the side stream ------------------------------------------
+    def launch_mix1(self, mix1: MixDesc, theta_prev: torch.Tensor) -> None:
+        """Start x = Mix1(theta_prev) on the side stream; returns immediately."""
+        if mix1.kind == FGD_MIX_IDENTITY:
+            raise ValueError("identity Mix1 needs no transfer: pass it as mix1_fused to step()")
+        ready = torch.cuda.current_stream(self.device).record_event()
+        self.side.wait_event(ready)
+        if mix1.kind == FGD_MIX_MEAN:
+            if self._x_vec is None:
+                self._x_vec = torch.empty(self.P, dtype=torch.float32, device=self.device)
+            x, is_vec = self._x_vec, True
+        else:
+            if self._x_mat is None:
+                self._x_mat = torch.empty((self.K, self.ld), dtype=torch.float32, device=self.device)
+            x, is_vec = self._x_mat, False
+        fgd_mix(self.ctx, mix1, theta_prev, x, out_is_vector=is_vec, stream=self.side)
+        self._pending = (self.side.record_event(), x, is_vec)
+
+    # ---- blocking part: wait for Mix1, then the fused outer step ---------------------------
+    def step(self, mix2: MixDesc, theta_local, theta_prev, momentum, theta_new, lr: float = 0.7,
+             mu: float = 0.9, mix1_fused: Optional[MixDesc] = None, want_cd: bool = True) -> None:
+        """Fused outer step on the current stream.  Uses the pending side-stream Mix1 result,
+        or computes Mix1 inside the kernel when ``mix1_fused`` is given."""
+        cd = self.cd_sumsq if want_cd else None
+        if mix1_fused is not None:
+            fgd_outer_step(self.ctx, mix2, mix1_fused, None, False, theta_local, theta_prev, momentum,
+                           theta_new, lr, mu, cd)
+            return
+        if self._pending is None:
+            raise RuntimeError("no Mix1 in flight: call launch_mix1() first or pass mix1_fused")
+        ev, x, is_vec = self._pending
+        self._pending = None
+        torch.cuda.current_stream(self.device).wait_event(ev)
+        fgd_outer_step(self.ctx, mix2, None, x, is_vec, theta_local, theta_prev, momentum, theta_new,
+                       lr, mu, cd)
+        # the side stream may not overwrite x for the next round before this kernel has read it
+        self.side.wait_event(torch.cuda.current_stream(self.device).record_event())
+
+    def consensus(self, theta) -> torch.Tensor:
+        fgd_consensus_distance(self.ctx, theta, self.cd_sumsq)
+        return self.cd_sumsq
+
+    def close(self):
+        self.ctx.close()

@@ -1,0 +1,311 @@
+"""GPU parity: every C-ABI entry point against the float64 oracle on the same seeded inputs.
+
+Bar: indices and edge masks bit-exact (checked in make_mix), fp32 parameters within max relative
+error 1e-5 (absolute 1e-7 near zero), consensus sums within relative 1e-5.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2606_22768_b200 as fgd
+from fgd_inputs import gen
+from tests.gpu_util import (Scenario, assert_cd_close, assert_param_close, check_padding, make_mix,
+                            padded, upload)
+
+pytestmark = pytest.mark.gpu
+
+SINK64 = gen.sinkhorn_W(0, 64)
+
+
+def _inputs(K, P, seed=0, worker_std=5e-4, sigma=1e-3):
+    tp = gen.theta0(seed, K, P, 0.02, worker_std)
+    tl = gen.local_params(tp, [sigma] * K, seed, 0)
+    v = gen.scaled_normal(seed, gen.TENSOR_MOMENTUM, 0, K, P, 1e-3)
+    return tp, tl, v
+
+
+# ------------------------------------------------------------------ fgd_outer_grad
+@pytest.mark.parametrize("K,P,ld", [(4, 1 << 20, None), (16, 100003, 100003), (3, 4100, 4352), (1, 1, 1), (64, 777, 780)])
+def test_outer_grad(K, P, ld):
+    ld = P if ld is None else ld
+    tp, tl, _ = _inputs(K, P)
+    f_tp, _ = upload(tp, ld)
+    f_tl, _ = upload(tl, ld)
+    f_g, g = padded(K, P, ld)
+    ctx = fgd.Context(K, P, ld)
+    fgd.fgd_outer_grad(ctx, f_tp, f_tl, f_g)
+    torch.cuda.synchronize()
+    ref = oracle.outer_grad(tp, tl)
+    # a single fp32 subtraction of fp32 inputs is correctly rounded: must equal the rounded oracle
+    assert np.array_equal(g.cpu().numpy(), ref.astype(np.float32))
+    check_padding(f_g, P, "g")
+    assert ctx.launch_count == 1
+
+
+# ------------------------------------------------------------------ fgd_mix
+MIX_CASES = [
+    (4, 1 << 18, ("mean",)), (4, 70001, ("ring",)), (8, 50000, ("xor",)), (16, 33333, ("hypercube",)),
+    (16, 40960, ("hypercube", 0.3)), (16, 5000, ("ring", 0.2, fgd.FGD_RENORM_SELF_ABSORB)),
+    (16, 20000, ("matching",)), (9, 3000, ("matching",)), (5, 12345, ("ring",)), (3, 999, ("mean",)),
+    (32, 20002, ("hypercube", 0.1)), (64, 10000, ("dense", SINK64)), (64, 4097, ("ring",)),
+    (16, 8192, ("dense", gen.sinkhorn_W(1, 16))), (7, 2048, ("dense", gen.sinkhorn_W(2, 7))),
+    (2, 1000, ("ring",)), (1, 100, ("identity",)), (8, 1000, ("identity",)),
+]
+
+
+@pytest.mark.parametrize("K,P,spec", MIX_CASES)
+def test_mix_matrix_output(K, P, spec):
+    x = gen.theta0(3, K, P, 0.02, 5e-3)
+    desc, W = make_mix(spec, K, 1, 3, 1)
+    ld = P + (4 - P % 4) % 4 + 4
+    f_in, _ = upload(x, ld)
+    f_out, out = padded(K, P, ld)
+    ctx = fgd.Context(K, P, ld)
+    fgd.fgd_mix(ctx, desc, f_in, f_out)
+    torch.cuda.synchronize()
+    assert_param_close(out, oracle.mix(W, x), f"mix {spec[0]} K={K}")
+    check_padding(f_out, P, "mix out")
+    # in place gives the same bits
+    fgd.fgd_mix(ctx, desc, f_in, f_in)
+    torch.cuda.synchronize()
+    assert torch.equal(f_in[:, :P], out)
+
+
+@pytest.mark.parametrize("K,P", [(4, 1 << 20), (16, 30001), (6, 513), (64, 4096)])
+def test_mix_mean_vector_output(K, P):
+    x = gen.theta0(4, K, P, 0.02, 5e-3)
+    f_in, _ = upload(x, P)
+    out = torch.full((P + 8,), -777.0, dtype=torch.float32, device="cuda")
+    ctx = fgd.Context(K, P)
+    fgd.fgd_mix(ctx, fgd.MixDesc.mean(K), f_in, out, out_is_vector=True)
+    torch.cuda.synchronize()
+    assert_param_close(out[:P], oracle.mix(oracle.dense_W("mean", K), x)[0], "mean vector")
+    assert bool((out[P:] == -777.0).all())
+
+
+# ------------------------------------------------------------------ fgd_consensus_distance
+@pytest.mark.parametrize("K,P,ld", [(4, 1 << 20, None), (16, 100001, 100004), (64, 20000, 20000), (32, 30002, 30002),
+                                     (5, 7777, 7780), (1, 50, 50), (2, 3, 4)])
+def test_consensus_distance(K, P, ld):
+    ld = P if ld is None else ld
+    th = gen.theta0(5, K, P, 0.02, 7e-4)
+    f_th, _ = upload(th, ld)
+    s = torch.full((K,), -1.0, dtype=torch.float64, device="cuda")
+    ctx = fgd.Context(K, P, ld)
+    fgd.fgd_consensus_distance(ctx, f_th, s)
+    torch.cuda.synchronize()
+    ref = oracle.consensus_sumsq(th)
+    assert_cd_close(s, ref, P, "consensus")
+    got = fgd.fgd_cd_finalize(s.cpu().numpy())
+    exp = oracle.cd_finalize(ref)
+    assert got[0] == pytest.approx(exp[0], rel=1e-5, abs=1e-9) and got[1] == pytest.approx(exp[1], rel=1e-5, abs=1e-12)
+    # deterministic: a second call gives the same bits
+    s2 = torch.zeros_like(s)
+    fgd.fgd_consensus_distance(ctx, f_th, s2)
+    torch.cuda.synchronize()
+    assert torch.equal(s, s2)
+
+
+# ------------------------------------------------------------------ fgd_outer_step, single call
+STEP_CASES = [
+    # K, P, mix1, mix2
+    (4, 1 << 18, ("mean",), ("ring",)),
+    (8, 60001, ("mean",), ("xor",)),
+    (16, 50000, ("mean",), ("ring",)),
+    (16, 30003, ("hypercube", 0.2), ("hypercube", 0.2)),
+    (16, 20000, ("matching",), ("matching",)),
+    (16, 8000, ("identity",), ("mean",)),
+    (16, 8000, ("mean",), ("identity",)),
+    (64, 9000, ("mean",), ("dense", SINK64)),
+    (64, 4100, ("mean",), ("hypercube",)),
+    (32, 10002, ("ring",), ("ring", 0.3)),
+    (16, 6000, ("mean",), ("dense", gen.sinkhorn_W(1, 16))),
+    (6, 5001, ("ring",), ("dense", gen.sinkhorn_W(2, 6))),
+    (5, 3000, ("mean",), ("ring",)),
+    (3, 2000, ("matching",), ("mean",)),
+    (2, 1000, ("mean",), ("ring",)),
+    (1, 300, ("identity",), ("identity",)),
+]
+
+
+@pytest.mark.parametrize("K,P,mix1,mix2", STEP_CASES)
+@pytest.mark.parametrize("mode", ["x_given", "mix1_fused"])
+def test_outer_step_single_call(K, P, mix1, mix2, mode):
+    if mode == "x_given" and mix1[0] == "identity":
+        pytest.skip("identity Mix1 has no transfer")
+    if mode == "mix1_fused" and mix1[0] == "dense":
+        pytest.skip("dense Mix1 is not fused")
+    tp, tl, v = _inputs(K, P, seed=7)
+    d1, W1 = make_mix(mix1, K, 2, 7, 1)
+    d2, W2 = make_mix(mix2, K, 2, 7, 2)
+    ld = P + (4 - P % 4) % 4
+    f_tp, g_tp = upload(tp, ld)
+    f_tl, _ = upload(tl, ld)
+    f_v, g_v = upload(v, ld)
+    f_new, g_new = padded(K, P, ld)
+    cd = torch.zeros(K, dtype=torch.float64, device="cuda")
+    ctx = fgd.Context(K, P, ld)
+    if mode == "x_given":
+        vec = mix1[0] == "mean"
+        x = torch.empty(P if vec else (K, ld), dtype=torch.float32, device="cuda")
+        fgd.fgd_mix(ctx, d1, f_tp, x, out_is_vector=vec)
+        fgd.fgd_outer_step(ctx, d2, None, x, vec, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+    else:
+        fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+    torch.cuda.synchronize()
+    ref_t, ref_v = oracle.outer_round(W1, W2, tp, tl, v, 0.7, 0.9)
+    assert_param_close(g_new, ref_t, "theta_new")
+    assert_param_close(g_v, ref_v, "momentum")
+    assert_cd_close(cd, oracle.consensus_sumsq(ref_t), P, "fused cd")
+    assert torch.equal(g_tp.cpu(), torch.from_numpy(tp)), "theta_prev must not change out of place"
+    for full, name in ((f_new, "theta_new"), (f_v, "momentum")):
+        check_padding(full, P, name)
+    # in place (theta_new == theta_prev), no consensus output: same bits as out of place
+    f_v2, g_v2 = upload(v, ld)
+    if mode == "x_given":
+        fgd.fgd_outer_step(ctx, d2, None, x, vec, f_tl, f_tp, f_v2, f_tp, 0.7, 0.9, None)
+    else:
+        fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v2, f_tp, 0.7, 0.9, None)
+    torch.cuda.synchronize()
+    assert torch.equal(g_tp, g_new) and torch.equal(g_v2, g_v)
+
+
+def test_outer_step_unaligned_pointers_take_the_elementwise_path():
+    K, P = 16, 5003
+    tp, tl, v = _inputs(K, P, seed=9)
+    d1, W1 = make_mix(("mean",), K, 0, 9, 1)
+    d2, W2 = make_mix(("ring",), K, 0, 9, 2)
+    ld = P + 2
+    bufs = [torch.full((K * ld + 1,), -777.0, dtype=torch.float32, device="cuda") for _ in range(4)]
+    views = [b[1:].view(K, ld) for b in bufs]  # base pointer 4 bytes off a 16-byte boundary
+    for view, a in zip(views[:3], (tp, tl, v)):
+        view[:, :P].copy_(torch.from_numpy(a))
+    ctx = fgd.Context(K, P, ld)
+    fgd.fgd_outer_step(ctx, d2, d1, None, False, views[1], views[0], views[2], views[3], 0.7, 0.9, None)
+    torch.cuda.synchronize()
+    ref_t, ref_v = oracle.outer_round(W1, W2, tp, tl, v, 0.7, 0.9)
+    assert_param_close(views[3][:, :P], ref_t, "theta_new")
+    assert_param_close(views[2][:, :P], ref_v, "momentum")
+    assert bool((views[3][:, P:] == -777.0).all()) and float(bufs[3][0]) == -777.0
+
+
+def test_lr_mu_are_honoured():
+    K, P = 4, 4096
+    tp, tl, v = _inputs(K, P, seed=11)
+    d1, W1 = make_mix(("ring",), K, 0, 11, 1)
+    d2, W2 = make_mix(("mean",), K, 0, 11, 2)
+    for lr, mu in ((1.0, 0.0), (0.3, 0.5)):
+        f_tp, _ = upload(tp, P)
+        f_tl, _ = upload(tl, P)
+        f_v, g_v = upload(v, P)
+        f_new, g_new = padded(K, P, P)
+        fgd.fgd_outer_step(fgd.Context(K, P), d2, d1, None, False, f_tl, f_tp, f_v, f_new, lr, mu, None)
+        torch.cuda.synchronize()
+        ref_t, ref_v = oracle.outer_round(W1, W2, tp, tl, v, lr, mu)
+        assert_param_close(g_new, ref_t, f"theta_new lr={lr}")
+        assert_param_close(g_v, ref_v, f"momentum mu={mu}")
+
+
+# ------------------------------------------------------------------ multi-round scenarios (the configs, reduced P)
+def test_config1_full_size():
+    """K=4, P=2^20, Mix1 mean, Mix2 ring 1/3, one round, seed 0 -- every element compared."""
+    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0).run(1)
+    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0, worker_std=5e-4, mode="fused").run(1)
+
+
+def test_config2_reduced():
+    """K=8, one-peer XOR Mix2 over 10 rounds (P reduced to 2^17+37, ragged)."""
+    Scenario(8, (1 << 17) + 37, ("mean",), ("xor",), ld=(1 << 17) + 40, seed=0).run(10)
+
+
+def test_config3_reduced():
+    """K=16, per-worker drift scale U[5e-4, 2e-3], side-stream Mix1 mean, ring Mix2, 10 rounds."""
+    sig = gen.drift_sigmas(0, 16, 5e-4, 2e-3)
+    Scenario(16, 150000, ("mean",), ("ring",), seed=0, sigmas=sig).run(10)
+
+
+@pytest.mark.parametrize("mode", ["factored", "fused"])
+def test_config4_reduced(mode):
+    """K=16 hypercube gossip for both mixes, independent p=0.1 edge failures, Metropolis
+    renormalisation, 20 rounds, consensus distance every round."""
+    Scenario(16, 65536 + 12, ("hypercube", 0.1), ("hypercube", 0.1), seed=0, mode=mode).run(20)
+
+
+def test_config5_reduced():
+    """K=64 dense Sinkhorn Mix2, Mix1 mean, 5 rounds."""
+    Scenario(64, 40000, ("mean",), ("dense", SINK64), seed=0).run(5)
+
+
+def test_pairwise_gossip_presets():
+    """The paper's four (Mix1, Mix2) presets with random-matching pairwise gossip, 4 rounds each."""
+    for m1, m2 in ((("identity",), ("mean",)), (("matching",), ("matching",)), (("mean",), ("identity",)),
+                   (("mean",), ("matching",))):
+        Scenario(8, 20001, m1, m2, ld=20004, seed=3, in_place=False).run(4)
+
+
+def test_diloco_preset_reaches_exact_consensus():
+    s = Scenario(16, 30000, ("identity",), ("mean",), seed=1).run(3)
+    rows = s.g_new
+    assert torch.equal(rows[0], rows[7]) and torch.equal(rows[0], rows[15])
+    assert float(s.drv.cd_sumsq.max()) <= 1e-12 * 30000
+
+
+def test_nonzero_initial_momentum_and_odd_K():
+    Scenario(7, 9999, ("ring", 0.2), ("ring", 0.2), ld=10000, seed=5, v0_std=1e-3, worker_std=1e-3).run(3)
+    Scenario(32, 12346, ("mean",), ("hypercube", 0.05), seed=6, v0_std=1e-3).run(3)
+
+
+# ------------------------------------------------------------------ determinism, errors
+def test_outer_step_is_bitwise_deterministic():
+    K, P = 16, 200000
+    tp, tl, v = _inputs(K, P, seed=2)
+    d2, _ = make_mix(("hypercube", 0.1), K, 0, 2, 2)
+    outs = []
+    for _ in range(2):
+        f_tp, _ = upload(tp, P)
+        f_tl, _ = upload(tl, P)
+        f_v, _ = upload(v, P)
+        cd = torch.zeros(K, dtype=torch.float64, device="cuda")
+        fgd.fgd_outer_step(fgd.Context(K, P), d2, fgd.MixDesc.mean(K), None, False, f_tl, f_tp, f_v, f_tp, 0.7, 0.9, cd)
+        torch.cuda.synchronize()
+        outs.append((f_tp.clone(), f_v.clone(), cd.clone()))
+    assert all(torch.equal(a, b) for a, b in zip(*outs))
+
+
+def test_argument_errors():
+    K, P = 4, 1024
+    ctx = fgd.Context(K, P)
+    a = torch.zeros((K, P), device="cuda")
+    b, c, d = torch.zeros_like(a), torch.zeros_like(a), torch.zeros_like(a)
+    ring = fgd.MixDesc.ring(K)
+    with pytest.raises(fgd.FgdError) as e:
+        fgd.fgd_outer_grad(ctx, a, b, a)
+    assert e.value.status == fgd.FGD_ERR_ALIAS
+    with pytest.raises(fgd.FgdError) as e:   # momentum aliases theta_local
+        fgd.fgd_outer_step(ctx, ring, fgd.MixDesc.mean(K), None, False, b, a, b, d)
+    assert e.value.status == fgd.FGD_ERR_ALIAS
+    with pytest.raises(fgd.FgdError) as e:   # partial overlap of theta_new and theta_prev
+        big = torch.zeros(K * P + 8, device="cuda")
+        fgd.fgd_outer_step(ctx, ring, fgd.MixDesc.mean(K), None, False, b, big[:K * P].view(K, P), c,
+                           big[4:K * P + 4].view(K, P))
+    assert e.value.status == fgd.FGD_ERR_ALIAS
+    with pytest.raises(fgd.FgdError) as e:   # neither x nor mix1_fused
+        fgd.fgd_outer_step(ctx, ring, None, None, False, b, a, c, d)
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:   # descriptor for another K
+        fgd.fgd_mix(ctx, fgd.MixDesc.ring(8), a, b)
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG and "does not match" in e.value.message
+    with pytest.raises(fgd.FgdError) as e:   # vector output only for the mean
+        fgd.fgd_mix(ctx, ring, a, b[0], out_is_vector=True)
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:
+        fgd.fgd_outer_step(ctx, ring, fgd.MixDesc.dense(np.eye(K)), None, False, b, a, c, d)
+    assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+    with pytest.raises(fgd.FgdError):
+        fgd.Context(65, 10)
+    with pytest.raises(fgd.FgdError):
+        fgd.Context(4, 10, ld=8)
+    # the context is still usable after errors
+    fgd.fgd_outer_grad(ctx, a, b, c)
+    torch.cuda.synchronize()
