@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the outer synchronisation round (one JSON line on stdout).
+
+A "step" is one whole outer round of the headline workload (K=16 workers, P=300M fp32
+parameters each): per-round mix descriptors built on the host, Mix1 = global average launched
+on a side stream, then on the main stream the fused outer step (outer gradient + ring Mix2 +
+Nesterov update + consensus partial sums) updating theta and the momentum in place, with the
+per-round consensus sums kept in a device log.  theta_local (the result of the workers' inner
+steps) is the step's input and is resident in HBM when the timed region starts.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1..5]
+
+N > 1 (launched by torch.distributed.run, one rank per GPU) runs N independent replicas of the
+same workload -- the path has no exchange between GPUs -- and reports the aggregate.
+--impl reference times the float64 CPU oracle on a bounded column sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "outer_round_worker_params_per_s"
+UNIT = "worker-params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# BASELINE.json configs (index = position in "configs", 1-based here)
+CONFIGS = {
+    1: dict(K=4, P=1 << 20, mix1=("mean",), mix2=("ring",), sig=(1e-3, 1e-3), p_fail=0.0,
+            name="cfg1 K=4 P=2^20 Mix1=mean Mix2=ring"),
+    2: dict(K=8, P=150_000_000, mix1=("mean",), mix2=("xor",), sig=(1e-3, 1e-3), p_fail=0.0,
+            name="cfg2 K=8 P=150M Mix1=mean Mix2=one-peer-xor"),
+    3: dict(K=16, P=300_000_000, mix1=("mean",), mix2=("ring",), sig=(5e-4, 2e-3), p_fail=0.0,
+            name="cfg3 K=16 P=300M Mix1=mean(side stream) Mix2=ring"),
+    4: dict(K=16, P=300_000_000, mix1=("hypercube",), mix2=("hypercube",), sig=(1e-3, 1e-3), p_fail=0.1,
+            name="cfg4 K=16 P=300M Mix1=Mix2=hypercube gossip, p_fail=0.1 Metropolis"),
+    5: dict(K=64, P=50_000_000, mix1=("mean",), mix2=("dense",), sig=(1e-3, 1e-3), p_fail=0.0,
+            name="cfg5 K=64 P=50M Mix1=mean Mix2=dense Sinkhorn"),
+}
+
+# DRAM bytes per worker-parameter of the fused outer-step kernel measured with ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum over one launch / (K*P) of that launch); the
+# capture it comes from is summarised under profiles/.  None = not captured yet.
+NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------- mixes per round
+def mix_desc(fgd, spec, cfg, rnd, seed, mix_id, dense_W):
+    K = cfg["K"]
+    kind = spec[0]
+    if kind == "mean":
+        return fgd.MixDesc.mean(K)
+    if kind == "identity":
+        return fgd.MixDesc.identity(K)
+    if kind == "dense":
+        return fgd.MixDesc.dense(dense_W)
+    d = {"ring": lambda: fgd.MixDesc.ring(K), "xor": lambda: fgd.MixDesc.onepeer_xor(K, rnd),
+         "hypercube": lambda: fgd.MixDesc.hypercube(K)}[kind]()
+    if cfg["p_fail"] > 0.0:
+        d = d.with_failures(seed, rnd, mix_id, cfg["p_fail"], fgd.FGD_RENORM_METROPOLIS)
+    return d
+
+
+# ---------------------------------------------------------------------- clocks sampling
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------- CPU oracle leg
+def oracle_leg(cfg, steps, warmup, seed=0, sample_cols=1 << 23):
+    """Times the float64 oracle, as it stands, on a bounded column sample of the workload."""
+    import oracle
+    from fgd_inputs import gen
+    from oracle import topology as T
+    K = cfg["K"]
+    Ps = min(cfg["P"], sample_cols)
+    sig = gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1] else np.full(K, cfg["sig"][0], np.float32)
+    theta = gen.theta0(seed, K, Ps).astype(np.float64)
+    v = np.zeros((K, Ps))
+    dense = gen.sinkhorn_W(seed, K).astype(np.float64) if "dense" in (cfg["mix1"][0], cfg["mix2"][0]) else None
+
+    def W_of(spec, rnd, mix_id):
+        kind = spec[0]
+        if kind in ("mean", "identity"):
+            return oracle.dense_W(kind, K)
+        if kind == "dense":
+            return dense
+        nbr, w, ws = {"ring": lambda: T.ring(K), "xor": lambda: T.onepeer_xor(K, rnd),
+                      "hypercube": lambda: T.hypercube(K)}[kind]()
+        mask, renorm = None, T.RENORM_NONE
+        if cfg["p_fail"] > 0.0:
+            mask, renorm = T.edge_mask(seed, rnd, mix_id, cfg["p_fail"], nbr), T.RENORM_METROPOLIS
+        return np.array(T.dense_from_sparse(nbr, *T.effective_weights(nbr, w, ws, mask, renorm)))
+
+    times = []
+    for r in range(warmup + steps):
+        local = theta + gen.scaled_normal(seed, gen.TENSOR_DRIFT, r, K, Ps, sig).astype(np.float64)
+        t0 = time.perf_counter()
+        W1, W2 = W_of(cfg["mix1"], r, 1), W_of(cfg["mix2"], r, 2)
+        theta, v = oracle.outer_round(W1, W2, theta, local, v, 0.7, 0.9)
+        oracle.consensus_sumsq(theta)
+        if r >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = sum(times) / len(times)
+    return {"value": K * Ps / sec, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {Ps} of {cfg['P']} columns, all K={K} workers, {len(times)} round(s), "
+                      f"{sec:.3f} s per round (round arithmetic + consensus sums only)"}, sec
+
+
+def run_reference(args):
+    cfg = CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = max(1, min(args.steps, 3)), max(0, min(args.warmup, 1))
+    base, sec = oracle_leg(cfg, steps, warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg["name"], "note": "CPU oracle on a bounded column sample; steps/warmup clamped"},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2606_22768_b200 as fgd
+    from fgd_inputs import gen, gpu as inputs_gpu
+    from paper_2606_22768_b200.round import OuterRound
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = CONFIGS[args.config]
+    K, P, seed = cfg["K"], cfg["P"], 0
+    steps, warmup = args.steps, max(args.warmup, 3)
+    sig = gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1] else np.full(K, cfg["sig"][0], np.float32)
+    dense_W = gen.sinkhorn_W(seed, K) if "dense" in (cfg["mix1"][0], cfg["mix2"][0]) else None
+
+    theta = torch.empty((K, P), dtype=torch.float32, device=dev)
+    local = torch.empty_like(theta)
+    mom = torch.zeros_like(theta)
+    inputs_gpu.theta0(theta, seed)
+    inputs_gpu.local_steps(local, theta, sig, seed, 0)
+    drv = OuterRound(K, P, device=local_rank)
+    cd_log = torch.zeros((warmup + steps + 8, K), dtype=torch.float64, device=dev)
+    main = torch.cuda.current_stream(dev)
+
+    def one_round(r, ev_pair=None):
+        m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
+        m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
+        drv.cd_sumsq = cd_log[r]
+        drv.launch_mix1(m1, theta)
+        if ev_pair is not None:
+            main.wait_event(drv._pending[0])     # keep the Mix1 wait out of the kernel's event pair
+            ev_pair[0].record(main)
+        drv.step(m2, local, theta, mom, theta, 0.7, 0.9)
+        if ev_pair is not None:
+            ev_pair[1].record(main)
+
+    for r in range(warmup):
+        one_round(r)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = drv.ctx.launch_count
+    t_begin.record(main)
+    for i in range(steps):
+        one_round(warmup + i, pairs[i])
+    t_end.record(main)
+    torch.cuda.synchronize()
+    launches = drv.ctx.launch_count - launches0
+    elapsed_ms = t_begin.elapsed_time(t_end)
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs)
+
+    ms_per_step = elapsed_ms / steps
+    units = K * P * world
+    value = units / (ms_per_step * 1e-3)
+    x_vec = cfg["mix1"][0] == "mean"
+    step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
+    mix1_bytes = (4 * K * P + 4 * P) if x_vec else 8 * K * P
+    peak, peak_kind = measured_peak()
+    achieved = step_bytes / (kern_ms * 1e-3) / 1e9
+    tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None if tr is None else tr * K * P, "kernel": "outer_step_kernel",
+                "kernel_ms": kern_ms, "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8000": achieved / 8000.0}
+
+    # consensus distance of the last round (both of the paper's definitions)
+    cd_norm, cd_sq = fgd.fgd_cd_finalize(cd_log[warmup + steps - 1].cpu().numpy())
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg["name"], "K": K, "P": P, "rounds_timed": steps,
+                       "l2": (f"inputs {(3 * K * P * 4) / 1e9:.1f} GB per round, larger than the 126 MB L2"
+                              if 3 * K * P * 4 > 4 * 126e6 else "working set fits in L2: latency config, not an HBM number"),
+                       "replicas": world, "step": "host mix build + side-stream Mix1 + fused outer step with consensus sums"},
+            "hbm_gbs_whole_step": (step_bytes + mix1_bytes) / (ms_per_step * 1e-3) / 1e9,
+            "roofline": roofline, "gpu_launches": int(launches), "clocks": clocks,
+            "consensus": {"cd_norm": cd_norm, "cd_sq": cd_sq}}
+
+    if rank == 0 and not args.no_overlap:
+        line["overlap"] = overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, dense_W)
+    if not args.no_e2e:
+        line["e2e"] = e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W, world, dev)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        del theta, local, mom
+        line["cpu_baseline"] = oracle_leg(cfg, 4, 1)[0]
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, dense_W, reps=3):
+    """Algorithm 1's overlap on one GPU: Mix1 on the side stream while a stand-in compute kernel
+    (the seeded drift generator) produces theta_local on the main stream.  Reports each alone
+    and both together; on one GPU they share HBM, so this models the dependency structure."""
+    dev = theta.device
+    main = torch.cuda.current_stream(dev)
+    m1 = mix_desc(fgd, cfg["mix1"], cfg, 0, seed, 1, dense_W)
+
+    def timed(fn):
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(main)
+            fn()
+            b.record(main)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return min(ts)
+
+    def mix1_only():
+        drv.launch_mix1(m1, theta)
+        main.wait_event(drv._pending[0])
+
+    def standin_only():
+        inputs_gpu.local_steps(local, theta, sig, seed, 1)
+
+    def both():
+        drv.launch_mix1(m1, theta)
+        inputs_gpu.local_steps(local, theta, sig, seed, 1)
+        main.wait_event(drv._pending[0])
+
+    out = {"mix1_alone_ms": timed(mix1_only), "standin_compute_alone_ms": timed(standin_only),
+           "overlapped_ms": timed(both)}
+    drv._pending = None
+    return out
+
+
+def e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W, world, dev, steps=3):
+    """Same round with theta_local arriving from pinned HOST memory every step and the consensus
+    sums read back to the host every step (both inside the timed region)."""
+    K, P = cfg["K"], cfg["P"]
+    host_local = torch.empty((K, P), dtype=torch.float32, pin_memory=True)
+    host_local.copy_(local)
+    host_cd = torch.empty(K, dtype=torch.float64, pin_memory=True)
+    main = torch.cuda.current_stream(dev)
+
+    def one(r):
+        m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
+        m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
+        drv.cd_sumsq = cd_log[0]
+        drv.launch_mix1(m1, theta)                       # overlaps the host-to-device copy
+        local.copy_(host_local, non_blocking=True)
+        drv.step(m2, local, theta, mom, theta, 0.7, 0.9)
+        host_cd.copy_(cd_log[0], non_blocking=True)
+        main.synchronize()
+
+    one(0)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(main)
+    for r in range(steps):
+        one(1 + r)
+    b.record(main)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": K * P * world / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": K * P * 4,
+            "d2h_bytes_per_step": K * 8, "steps": steps, "ms_per_step": ms / steps}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
