@@ -58,7 +58,7 @@ typedef enum {
   FGD_ERR_ALIAS = -3,       /* forbidden overlap between tensors */
   FGD_ERR_UNSUPPORTED = -4, /* valid request this build has no kernel for */
   FGD_ERR_CUDA = -5,        /* a CUDA runtime call failed (message holds the CUDA error) */
-  FGD_ERR_TIMEOUT = -6      /* reserved for bounded device-side waits */
+  FGD_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (see fgd_device_status) */
 } fgd_status;
 
 typedef struct fgd_ctx fgd_ctx; /* opaque; owns O(#CTAs * K) doubles of device scratch */
@@ -71,6 +71,16 @@ int fgd_destroy(fgd_ctx* ctx);
  * last failing fgd_create / host helper on this thread.  The string is owned by the library. */
 const char* fgd_last_error(const fgd_ctx* ctx);
 const char* fgd_status_string(int status);
+/* Which kernel family fgd_outer_step uses.  AUTO (default): the TMA-pipelined kernel when the
+ * tensors allow it (16-byte aligned bases, ld % 4 == 0, two pipeline stages fit in shared
+ * memory), else the register kernel.  REGISTER / TMA force one (TMA fails with
+ * FGD_ERR_UNSUPPORTED when not eligible).  Both compute the same round. */
+typedef enum { FGD_PATH_AUTO = 0, FGD_PATH_REGISTER = 1, FGD_PATH_TMA = 2 } fgd_path;
+int fgd_set_path(fgd_ctx* ctx, int path);
+/* Synchronises `stream` and reports whether any kernel of this context abandoned a bounded
+ * device-side wait since the last check: FGD_OK, or FGD_ERR_TIMEOUT (then the outputs of the
+ * affected launch are invalid).  Clears the flag. */
+int fgd_device_status(fgd_ctx* ctx, void* stream);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t fgd_launch_count(const fgd_ctx* ctx);
 

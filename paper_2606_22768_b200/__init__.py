@@ -34,6 +34,7 @@ FGD_ERR_TIMEOUT = -6
 
 FGD_MIX_IDENTITY, FGD_MIX_MEAN, FGD_MIX_SPARSE, FGD_MIX_DENSE = 0, 1, 2, 3
 FGD_RENORM_NONE, FGD_RENORM_SELF_ABSORB, FGD_RENORM_METROPOLIS = 0, 1, 2
+FGD_PATH_AUTO, FGD_PATH_REGISTER, FGD_PATH_TMA = 0, 1, 2
 
 
 class FgdError(RuntimeError):
@@ -62,6 +63,8 @@ def _load():
         "fgd_last_error": (ctypes.c_char_p, [vp]),
         "fgd_status_string": (ctypes.c_char_p, [i32]),
         "fgd_launch_count": (i64, [vp]),
+        "fgd_set_path": (i32, [vp, i32]),
+        "fgd_device_status": (i32, [vp, vp]),
         "fgd_outer_grad": (i32, [vp, vp, vp, vp, vp]),
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
@@ -263,6 +266,15 @@ class Context:
     @property
     def launch_count(self) -> int:
         return int(_lib.fgd_launch_count(self._h))
+
+
+def fgd_set_path(ctx: Context, path: int) -> None:
+    ctx._check(_lib.fgd_set_path(ctx._h, int(path)))
+
+
+def fgd_device_status(ctx: Context, stream=None) -> None:
+    """Synchronises the stream; raises FgdError(FGD_ERR_TIMEOUT) if a device-side wait gave up."""
+    ctx._check(_lib.fgd_device_status(ctx._h, _stream(stream)))
 
 
 def fgd_outer_grad(ctx: Context, theta_prev, theta_local, g, stream=None) -> None:

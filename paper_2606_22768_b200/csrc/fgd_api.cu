@@ -7,6 +7,7 @@
 #include <utility>
 
 #include "fgd_kernels.cuh"
+#include "fgd_step_tma.cuh"
 
 using namespace fgd;
 
@@ -22,6 +23,10 @@ struct fgd_ctx {
   int64_t P = 0, ld = 0;
   int num_sms = 0;
   double* partials = nullptr;  // [kMaxPartialBlocks][K]
+  int* status = nullptr;       // device status word written by bounded waits that gave up
+  int path = FGD_PATH_AUTO;    // which fused-step kernel family to use
+  int max_smem_optin = 0;
+  void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
   int64_t launches = 0;
   char err[256] = "";
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
@@ -189,6 +194,87 @@ int launch_finalize(fgd_ctx* c, int nblocks, double* out, cudaStream_t st) {
   return check_launch(c, "consensus_finalize_kernel");
 }
 
+
+// ---- TMA-pipelined fused step ------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D map of a [K, ld] fp32 matrix restricted to its first P columns; box = boxc columns x K rows.
+// Columns at or beyond P read as zero.
+int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc) {
+  const cuuint64_t dims[2] = {(cuuint64_t)c->P, (cuuint64_t)c->K};
+  const cuuint64_t strides[1] = {(cuuint64_t)c->ld * sizeof(float)};
+  const cuuint32_t box[2] = {(cuuint32_t)boxc, (cuuint32_t)c->K};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(c, FGD_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return FGD_OK;
+}
+
+constexpr int kConsumers = 128;  // consumer threads per CTA of the TMA kernel (+ one producer warp)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Can the TMA kernel run this call?  Writes the vector width and stage count to use.
+bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, int* vec_out, int* stages_out) {
+  if (!c->encode_tiled) return false;
+  if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
+  if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
+  if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
+  const int K = c->K, KT = kt_of(K), NT = a.xsrc == XSRC_MATRIX ? 4 : 3;
+  const size_t fixed = 128 + 4096 + (dense2 ? sizeof(float) * K * K : 0) + (KT == 0 ? sizeof(float) * K * kConsumers : 0);
+  for (int vec = want_vec(KT); vec >= 1; vec >>= 1) {
+    if (c->P % vec != 0) continue;
+    if (vec > 1 && a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
+    const size_t stage = tma_stage_bytes(K, kConsumers * vec, NT);
+    if ((size_t)c->max_smem_optin < fixed + 2 * stage) continue;
+    int stages = (int)(((size_t)c->max_smem_optin - fixed) / stage);
+    if (stages > kMaxStages) stages = kMaxStages;
+    *vec_out = vec;
+    *stages_out = stages;
+    return true;
+  }
+  return false;
+}
+
+int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
+                    const GatherMix& g1, int vec, int stages, cudaStream_t st, int* grid_out) {
+  const int K = c->K, KT = kt_of(K);
+  TmaStepArgs ta;
+  ta.s = a;
+  ta.status = c->status;
+  ta.n_tensors = a.xsrc == XSRC_MATRIX ? 4 : 3;
+  ta.stages = stages;
+  const int T = kConsumers * vec;
+  const int boxc = T < 256 ? T : 256;
+  CUtensorMap tp, tl, tm, tx;
+  if (int rc = make_tensor_map(c, &tp, a.theta_prev, boxc)) return rc;
+  if (int rc = make_tensor_map(c, &tl, a.theta_local, boxc)) return rc;
+  if (int rc = make_tensor_map(c, &tm, a.momentum, boxc)) return rc;
+  if (int rc = make_tensor_map(c, &tx, a.xsrc == XSRC_MATRIX ? a.x : a.theta_prev, boxc)) return rc;
+  const size_t smem = 128 + tma_stage_bytes(K, T, ta.n_tensors) * stages + (dense2 ? sizeof(float) * K * K : 0) +
+                      (KT == 0 ? sizeof(float) * K * kConsumers : 0);
+  const int64_t ntiles = (c->P + T - 1) / T;
+  return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
+    int grid = 0;
+    if (dense2) {
+      auto kern = outer_step_tma_kernel<KTc, VECc, kConsumers, true, DenseMix>;
+      if (int r = persistent_grid(c, kern, kConsumers + 32, smem, ntiles, &grid)) return r;
+      kern<<<grid, kConsumers + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
+    } else {
+      auto kern = outer_step_tma_kernel<KTc, VECc, kConsumers, false, GatherMix>;
+      if (int r = persistent_grid(c, kern, kConsumers + 32, smem, ntiles, &grid)) return r;
+      kern<<<grid, kConsumers + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
+    }
+    *grid_out = grid;
+    return check_launch(c, "outer_step_tma_kernel");
+  });
+}
+
 }  // namespace
 
 extern "C" {
@@ -211,7 +297,17 @@ int fgd_create(fgd_ctx** out, int device, int K, int64_t P, int64_t ld) {
   c->P = P;
   c->ld = ld;
   e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
   if (e == cudaSuccess) e = cudaMalloc(&c->partials, sizeof(double) * (size_t)kMaxPartialBlocks * FGD_MAX_K);
+  if (e == cudaSuccess) e = cudaMalloc(&c->status, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
+  if (e == cudaSuccess) {
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      c->encode_tiled = nullptr;  // the TMA path is then unavailable; the register path still works
+    cudaGetLastError();
+  }
   if (e != cudaSuccess) {
     int rc = cuda_fail(nullptr, e, "fgd_create");
     delete c;
@@ -225,11 +321,34 @@ int fgd_destroy(fgd_ctx* c) {
   if (!c) return FGD_OK;
   DeviceGuard guard(c->device);
   cudaError_t e = cudaFree(c->partials);
+  cudaFree(c->status);
   delete c;
   return e == cudaSuccess ? FGD_OK : cuda_fail(nullptr, e, "fgd_destroy");
 }
 
 const char* fgd_last_error(const fgd_ctx* c) { return c ? c->err : g_thread_error; }
+
+int fgd_set_path(fgd_ctx* c, int path) {
+  if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_set_path: ctx is NULL");
+  if (path < FGD_PATH_AUTO || path > FGD_PATH_TMA) return fail(c, FGD_ERR_INVALID_ARG, "fgd_set_path: unknown path %d", path);
+  c->path = path;
+  return FGD_OK;
+}
+
+int fgd_device_status(fgd_ctx* c, void* stream) {
+  if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_device_status: ctx is NULL");
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return fail(c, FGD_ERR_CUDA, "cannot select device %d", c->device);
+  int h = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FGD_CUDA(c, cudaMemcpyAsync(&h, c->status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  FGD_CUDA(c, cudaStreamSynchronize(st));
+  if (h != 0) {
+    FGD_CUDA(c, cudaMemsetAsync(c->status, 0, sizeof(int), st));
+    return fail(c, h, "a device-side wait gave up (status %d); results of that launch are invalid", h);
+  }
+  return FGD_OK;
+}
 int64_t fgd_launch_count(const fgd_ctx* c) { return c ? c->launches : 0; }
 
 int fgd_outer_grad(fgd_ctx* c, const float* theta_prev, const float* theta_local, float* g, void* stream) {
@@ -356,27 +475,36 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
   else if (int rc = make_gather(c, mix2, &g2)) return rc;
 
   const int KT = kt_of(K);
-  const int vec = pick_vec(want_vec(KT), c->P, c->ld,
-                           {theta_local, theta_prev, momentum, theta_new, x});
   int grid = 0;
-  int rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
-    const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
-    const size_t col = sizeof(float) * (size_t)K * kBlock * VECc;
-    size_t smem = col + (a.stage_tp ? col : 0);
-    if (dense2) {
-      if (!StepTraits<KTc, VECc, true>::kRegArrays) smem += col + sizeof(float) * (size_t)K * kBlock;
-      smem += sizeof(float) * (size_t)K * K;
-      auto kern = outer_step_kernel<KTc, VECc, true, kBlock, DenseMix>;
-      if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
-      kern<<<grid, kBlock, smem, st>>>(a, d2, g1);
-    } else {
-      if (!StepTraits<KTc, VECc, false>::kRegArrays) smem += col + sizeof(float) * (size_t)K * kBlock;
-      auto kern = outer_step_kernel<KTc, VECc, false, kBlock, GatherMix>;
-      if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
-      kern<<<grid, kBlock, smem, st>>>(a, g2, g1);
-    }
-    return check_launch(c, "outer_step_kernel");
-  });
+  int rc = FGD_OK;
+  int tma_vec = 0, tma_stages = 0;
+  const bool can_tma = tma_eligible(c, a, dense2, &tma_vec, &tma_stages);
+  if (c->path == FGD_PATH_TMA && !can_tma)
+    return fail(c, FGD_ERR_UNSUPPORTED,
+                "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
+  if (can_tma && c->path != FGD_PATH_REGISTER) {
+    rc = launch_step_tma(c, a, dense2, g2, d2, g1, tma_vec, tma_stages, st, &grid);
+  } else {
+    const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x});
+    rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
+      const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
+      const size_t col = sizeof(float) * (size_t)K * kBlock * VECc;
+      size_t smem = col + (a.stage_tp ? col : 0);
+      if (dense2) {
+        if (!StepTraits<KTc, VECc, true>::kRegArrays) smem += col + sizeof(float) * (size_t)K * kBlock;
+        smem += sizeof(float) * (size_t)K * K;
+        auto kern = outer_step_kernel<KTc, VECc, true, kBlock, DenseMix>;
+        if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
+        kern<<<grid, kBlock, smem, st>>>(a, d2, g1);
+      } else {
+        if (!StepTraits<KTc, VECc, false>::kRegArrays) smem += col + sizeof(float) * (size_t)K * kBlock;
+        auto kern = outer_step_kernel<KTc, VECc, false, kBlock, GatherMix>;
+        if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
+        kern<<<grid, kBlock, smem, st>>>(a, g2, g1);
+      }
+      return check_launch(c, "outer_step_kernel");
+    });
+  }
   if (rc) return rc;
   if (cd_sumsq) return launch_finalize(c, grid, cd_sumsq, st);
   return FGD_OK;

@@ -1,0 +1,300 @@
+// Fused outer step, TMA-pipelined variant (the fast path on sm_100a).
+//
+// The register-only kernel keeps every load it has in flight in registers, which caps the
+// bytes in flight per SM well below what HBM3e needs.  Here one producer warp streams
+// [K rows x T columns] boxes of theta_prev, theta_local and the momentum (and the Mix1 result
+// when it is a matrix) into a ring of shared-memory stages with 2-D TMA loads
+// (cp.async.bulk.tensor) that complete on mbarriers, so a full stage or more (~100-190 KB per
+// SM) is always in flight regardless of register use.  Consumer threads each own VEC adjacent
+// columns of the tile and walk all K rows in shared memory: every cross-worker quantity
+// (neighbour gathers, column means) is thread-local, so consumers never synchronise with each
+// other -- only with the producer, through the stage's full / empty mbarriers.  Results are
+// streamed to HBM straight from registers.  Stage buffers are reused in place:
+//     A = theta_prev tile, B = theta_local tile -> outer gradient g, C = momentum tile -> theta_new.
+// Every mbarrier wait is bounded; on a timeout the kernel records FGD_ERR_TIMEOUT in the
+// status word, drains its own copies and returns.
+#ifndef FGD_STEP_TMA_CUH_
+#define FGD_STEP_TMA_CUH_
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "fgd_kernels.cuh"
+
+namespace fgd {
+
+constexpr uint32_t kSpinLimit = 1u << 24;  // try_wait iterations before a wait gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait for the phase with the given parity; false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
+      : "memory");
+}
+
+struct TmaStepArgs {
+  StepArgs s;
+  int* status;       // device status word (0 = ok)
+  int n_tensors;     // 3, or 4 when x is a [K, ld] matrix
+  int stages;        // pipeline depth, 2..kMaxStages
+};
+
+// Shared-memory need of the kernel (bytes), also used by the host to size the launch.
+__host__ __device__ inline size_t tma_stage_bytes(int K, int T, int n_tensors) {
+  return (size_t)n_tensors * K * T * sizeof(float);
+}
+
+constexpr int kMaxStages = 8;
+
+template <int KT, int VEC, int CONSUMERS, bool DENSE2, typename M2>
+__global__ void __launch_bounds__(CONSUMERS + 32)
+outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
+                      const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
+                      const __grid_constant__ CUtensorMap tm_mom, const __grid_constant__ CUtensorMap tm_x) {
+  constexpr int T = CONSUMERS * VEC;          // columns per tile
+  constexpr int BOXC = T < 256 ? T : 256;     // columns per TMA box (box extents are <= 256)
+  constexpr int NBOX = T / BOXC;              // boxes per tensor per tile
+  constexpr int TPB = BOXC / VEC;             // consumer threads per box
+  constexpr int NWARP = CONSUMERS / 32 + 1;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * kMaxStages];
+  __shared__ int abort_flag;
+  __shared__ double red[NWARP][FGD_MAX_K];
+
+  const StepArgs& a = ta.s;
+  const int K = KT > 0 ? KT : a.K;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool want_cd = a.partials != nullptr;
+  const int NT = ta.n_tensors;
+  const int STAGES = ta.stages;
+  const size_t tens_floats = (size_t)K * T;                 // one tensor's box in a stage
+  const size_t stage_floats = tens_floats * NT;
+  // TMA destinations must be 128-byte aligned: round the ring's start up (the launch adds 128 B)
+  float* stages = reinterpret_cast<float*>(smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u));
+  float* wts = stages + stage_floats * STAGES;              // dense Wt [K*K] (DENSE2 only)
+  float* sas = wts + (DENSE2 ? K * K : 0);                  // runtime-K consensus sums [K][CONSUMERS]
+
+  const int64_t P = a.P, ld = a.ld;
+  const int64_t ntiles = (P + T - 1) / T;
+  const size_t box_floats = (size_t)K * BOXC;               // one TMA box
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bars[s]), 1);                       // full: one expect_tx arrival
+      mbar_init(smem_u32(&bars[kMaxStages + s]), CONSUMERS);      // empty: every consumer arrives
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if constexpr (DENSE2) {
+    for (int i = tid; i < K * K; i += CONSUMERS + 32) wts[i] = m2.Wt[i];
+  }
+  __syncthreads();
+
+  constexpr int KR = KT > 0 ? KT : 1;
+  float sacc[KR];
+#pragma unroll
+  for (int m = 0; m < KR; ++m) sacc[m] = 0.f;
+
+  if (warp == CONSUMERS / 32) {
+    // ===================================================== producer warp (one elected lane)
+    if (lane == 0) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      int64_t i = 0;
+      bool ok = true;
+      for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
+        const int s = (int)(i % STAGES);
+        const uint32_t use = (uint32_t)(i / STAGES);
+        if (use > 0) ok = mbar_wait(smem_u32(&bars[kMaxStages + s]), (use - 1) & 1);
+        if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
+        const uint32_t full = smem_u32(&bars[s]);
+        const int64_t c0 = tile * T;
+        const int64_t left = P - c0;                                  // > 0
+        const int nbox = left >= T ? NBOX : (int)((left + BOXC - 1) / BOXC);   // boxes that touch the tensor
+        mbar_expect_tx(full, (uint32_t)(box_floats * sizeof(float)) * (uint32_t)(nbox * NT));
+        const uint32_t dst = smem_u32(stages + stage_floats * s);
+        for (int b = 0; b < nbox; ++b) {
+          const uint32_t d = dst + (uint32_t)(box_floats * sizeof(float)) * b;
+          const int c = (int)(c0 + (int64_t)b * BOXC);
+          tma_load_2d(d, &tm_prev, c, 0, full, policy);
+          tma_load_2d(d + (uint32_t)(tens_floats * 4), &tm_local, c, 0, full, policy);
+          tma_load_2d(d + (uint32_t)(tens_floats * 8), &tm_mom, c, 0, full, policy);
+          if (NT == 4) tma_load_2d(d + (uint32_t)(tens_floats * 12), &tm_x, c, 0, full, policy);
+        }
+      }
+      if (!ok) {
+        // give up: flag it, then wait (bounded) for every copy this thread still has in flight
+        *(volatile int*)&abort_flag = 1;
+        atomicExch(ta.status, FGD_ERR_TIMEOUT);
+        for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
+          mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1);
+      }
+    }
+  } else {
+    // ===================================================== consumers
+    if constexpr (KT == 0) {
+      for (int m = 0; m < K; ++m) sas[m * CONSUMERS + tid] = 0.f;
+    }
+    const float invK = 1.0f / (float)K;
+    const float lr = a.lr, mu = a.mu;
+    int64_t i = 0;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
+      const int s = (int)(i % STAGES);
+      const uint32_t use = (uint32_t)(i / STAGES);
+      const int64_t col = tile * T + (int64_t)tid * VEC;
+      const bool live = col < P;
+      Pack<VEC> xv;
+      if (a.xsrc == XSRC_VECTOR && live) xv = ld_stream<VEC>(a.x + col);   // latency hides behind the wait
+      if (!mbar_wait(smem_u32(&bars[s]), use & 1)) {
+        *(volatile int*)&abort_flag = 1;
+        atomicExch(ta.status, FGD_ERR_TIMEOUT);
+        break;
+      }
+      // this thread's box inside each tensor of the stage; within a box, element (m, t) of a
+      // [K][TPB] array of Pack<VEC>
+      float* A = stages + stage_floats * s + box_floats * (tid / TPB);   // theta_prev
+      float* B = A + tens_floats;              // theta_local -> g
+      float* C = B + tens_floats;              // momentum -> theta_new
+      float* X = C + tens_floats;              // Mix1 result (matrix), if staged
+      const int t = tid % TPB;
+      if (live) {
+        // ---- phase 1: outer gradients of all workers into B, column sums
+        Pack<VEC> gsum, tsum;
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) gsum.v[q] = tsum.v[q] = 0.f;
+#pragma unroll(KT > 0 ? KT : 4)
+        for (int m = 0; m < K; ++m) {
+          const Pack<VEC> tp = SCol<VEC>::ld(A, m * TPB + t);
+          const Pack<VEC> tl = SCol<VEC>::ld(B, m * TPB + t);
+          Pack<VEC> g;
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) {
+            g.v[q] = tp.v[q] - tl.v[q];
+            gsum.v[q] += g.v[q];
+            tsum.v[q] += tp.v[q];
+          }
+          SCol<VEC>::st(B, m * TPB + t, g);
+        }
+        if (a.xsrc != XSRC_VECTOR) {
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) xv.v[q] = tsum.v[q] * invK;   // fused mean Mix1
+        }
+        Pack<VEC> gmean, asum;
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) {
+          gmean.v[q] = gsum.v[q] * invK;
+          asum.v[q] = 0.f;
+        }
+        // ---- phase 2: mix, Nesterov step, stream out, keep theta_new in C
+        auto finish_row = [&](int m, const Pack<VEC>& gh) {
+          const size_t off = (size_t)m * ld + col;
+          Pack<VEC> xm;
+          if (a.xsrc == XSRC_MATRIX) xm = SCol<VEC>::ld(X, m * TPB + t);
+          else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) xm = gather_row<VEC, TPB>(m1, m, A, t);
+          else xm = xv;
+          const Pack<VEC> v = SCol<VEC>::ld(C, m * TPB + t);
+          Pack<VEC> vn, tn;
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) {
+            vn.v[q] = fmaf(mu, v.v[q], gh.v[q]);
+            tn.v[q] = xm.v[q] - lr * fmaf(mu, vn.v[q], gh.v[q]);
+            asum.v[q] += tn.v[q];
+          }
+          st_stream<VEC>(a.momentum + off, vn);
+          st_stream<VEC>(a.theta_new + off, tn);
+          if (want_cd) SCol<VEC>::st(C, m * TPB + t, tn);
+        };
+        if constexpr (DENSE2) {
+          dense_rows<KT, VEC, TPB, (KT > 0 && KT <= 16)>(K, wts, B, t, finish_row);
+        } else {
+#pragma unroll(KT > 0 ? KT : 2)
+          for (int m = 0; m < K; ++m) {
+            Pack<VEC> gh;
+            if (m2.kind == KMIX_MEAN) gh = gmean;
+            else gh = gather_row<VEC, TPB>(m2, m, B, t);
+            finish_row(m, gh);
+          }
+        }
+        // ---- phase 3: squared deviation of theta_new from its column mean
+        if (want_cd) {
+#pragma unroll(KT > 0 ? KT : 4)
+          for (int m = 0; m < K; ++m) {
+            const Pack<VEC> tv = SCol<VEC>::ld(C, m * TPB + t);
+            float sq = 0.f;
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) {
+              const float d = tv.v[q] - asum.v[q] * invK;
+              sq = fmaf(d, d, sq);
+            }
+            if constexpr (KT > 0) sacc[m] += sq;
+            else sas[m * CONSUMERS + tid] += sq;
+          }
+        }
+      }
+      // this thread's reads and writes of the stage are done: order them before the TMA refill
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&bars[kMaxStages + s]));
+    }
+  }
+
+  // ---- consensus partial sums of the CTA (deterministic order); the producer warp adds zeros
+  if (want_cd) {
+    const bool consumer = warp < CONSUMERS / 32;
+    if constexpr (KT > 0) {
+#pragma unroll
+      for (int m = 0; m < KT; ++m) {
+        double d = consumer ? (double)sacc[m] : 0.0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
+        if (lane == 0) red[warp][m] = d;
+      }
+    } else {
+      for (int m = 0; m < K; ++m) {
+        double d = consumer ? (double)sas[m * CONSUMERS + tid] : 0.0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
+        if (lane == 0) red[warp][m] = d;
+      }
+    }
+  }
+  __syncthreads();
+  if (want_cd && tid < K) {
+    double d = 0.0;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) d += red[w][tid];
+    a.partials[(size_t)blockIdx.x * K + tid] = d;
+  }
+}
+
+}  // namespace fgd
+#endif

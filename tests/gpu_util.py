@@ -93,7 +93,7 @@ class Scenario:
     compares theta_new, momentum and the consensus sums after every round."""
 
     def __init__(self, K, P, mix1, mix2, *, ld=None, seed=0, sigmas=1e-3, worker_std=0.0, mode="factored",
-                 in_place=True, lr=0.7, mu=0.9, v0_std=0.0):
+                 in_place=True, lr=0.7, mu=0.9, v0_std=0.0, path=fgd.FGD_PATH_AUTO):
         self.K, self.P, self.ld = K, P, P if ld is None else ld
         self.mix1, self.mix2, self.seed, self.mode, self.in_place = mix1, mix2, seed, mode, in_place
         self.lr, self.mu = lr, mu
@@ -107,6 +107,7 @@ class Scenario:
         self.full_loc, self.g_loc = padded(K, P, self.ld)
         self.full_new, self.g_new = (self.full_prev, self.g_prev) if in_place else padded(K, P, self.ld)
         self.drv = OuterRound(K, P, self.ld)
+        fgd.fgd_set_path(self.drv.ctx, path)
 
     def run(self, R):
         K, P = self.K, self.P
@@ -134,4 +135,5 @@ class Scenario:
                 check_padding(full, P, name)
             if not self.in_place:
                 self.g_prev.copy_(self.g_new)
+        fgd.fgd_device_status(self.drv.ctx)
         return self

@@ -16,6 +16,7 @@ from tests.gpu_util import (Scenario, assert_cd_close, assert_param_close, check
 pytestmark = pytest.mark.gpu
 
 SINK64 = gen.sinkhorn_W(0, 64)
+PATHS = [pytest.param(fgd.FGD_PATH_TMA, id="tma"), pytest.param(fgd.FGD_PATH_REGISTER, id="reg")]
 
 
 def _inputs(K, P, seed=0, worker_std=5e-4, sigma=1e-3):
@@ -131,7 +132,8 @@ STEP_CASES = [
 
 @pytest.mark.parametrize("K,P,mix1,mix2", STEP_CASES)
 @pytest.mark.parametrize("mode", ["x_given", "mix1_fused"])
-def test_outer_step_single_call(K, P, mix1, mix2, mode):
+@pytest.mark.parametrize("path", PATHS)
+def test_outer_step_single_call(K, P, mix1, mix2, mode, path):
     if mode == "x_given" and mix1[0] == "identity":
         pytest.skip("identity Mix1 has no transfer")
     if mode == "mix1_fused" and mix1[0] == "dense":
@@ -146,6 +148,7 @@ def test_outer_step_single_call(K, P, mix1, mix2, mode):
     f_new, g_new = padded(K, P, ld)
     cd = torch.zeros(K, dtype=torch.float64, device="cuda")
     ctx = fgd.Context(K, P, ld)
+    fgd.fgd_set_path(ctx, path)
     if mode == "x_given":
         vec = mix1[0] == "mean"
         x = torch.empty(P if vec else (K, ld), dtype=torch.float32, device="cuda")
@@ -169,6 +172,7 @@ def test_outer_step_single_call(K, P, mix1, mix2, mode):
         fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v2, f_tp, 0.7, 0.9, None)
     torch.cuda.synchronize()
     assert torch.equal(g_tp, g_new) and torch.equal(g_v2, g_v)
+    fgd.fgd_device_status(ctx)
 
 
 def test_outer_step_unaligned_pointers_take_the_elementwise_path():
@@ -182,6 +186,11 @@ def test_outer_step_unaligned_pointers_take_the_elementwise_path():
     for view, a in zip(views[:3], (tp, tl, v)):
         view[:, :P].copy_(torch.from_numpy(a))
     ctx = fgd.Context(K, P, ld)
+    fgd.fgd_set_path(ctx, fgd.FGD_PATH_TMA)
+    with pytest.raises(fgd.FgdError) as e:
+        fgd.fgd_outer_step(ctx, d2, d1, None, False, views[1], views[0], views[2], views[3], 0.7, 0.9, None)
+    assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+    fgd.fgd_set_path(ctx, fgd.FGD_PATH_AUTO)
     fgd.fgd_outer_step(ctx, d2, d1, None, False, views[1], views[0], views[2], views[3], 0.7, 0.9, None)
     torch.cuda.synchronize()
     ref_t, ref_v = oracle.outer_round(W1, W2, tp, tl, v, 0.7, 0.9)
@@ -208,33 +217,38 @@ def test_lr_mu_are_honoured():
 
 
 # ------------------------------------------------------------------ multi-round scenarios (the configs, reduced P)
-def test_config1_full_size():
+@pytest.mark.parametrize("path", PATHS)
+def test_config1_full_size(path):
     """K=4, P=2^20, Mix1 mean, Mix2 ring 1/3, one round, seed 0 -- every element compared."""
-    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0).run(1)
-    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0, worker_std=5e-4, mode="fused").run(1)
+    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0, path=path).run(1)
+    Scenario(4, 1 << 20, ("mean",), ("ring",), seed=0, worker_std=5e-4, mode="fused", path=path).run(1)
 
 
-def test_config2_reduced():
+@pytest.mark.parametrize("path", PATHS)
+def test_config2_reduced(path):
     """K=8, one-peer XOR Mix2 over 10 rounds (P reduced to 2^17+37, ragged)."""
-    Scenario(8, (1 << 17) + 37, ("mean",), ("xor",), ld=(1 << 17) + 40, seed=0).run(10)
+    Scenario(8, (1 << 17) + 37, ("mean",), ("xor",), ld=(1 << 17) + 40, seed=0, path=path).run(10)
 
 
-def test_config3_reduced():
+@pytest.mark.parametrize("path", PATHS)
+def test_config3_reduced(path):
     """K=16, per-worker drift scale U[5e-4, 2e-3], side-stream Mix1 mean, ring Mix2, 10 rounds."""
     sig = gen.drift_sigmas(0, 16, 5e-4, 2e-3)
-    Scenario(16, 150000, ("mean",), ("ring",), seed=0, sigmas=sig).run(10)
+    Scenario(16, 150000, ("mean",), ("ring",), seed=0, sigmas=sig, path=path).run(10)
 
 
 @pytest.mark.parametrize("mode", ["factored", "fused"])
-def test_config4_reduced(mode):
+@pytest.mark.parametrize("path", PATHS)
+def test_config4_reduced(mode, path):
     """K=16 hypercube gossip for both mixes, independent p=0.1 edge failures, Metropolis
     renormalisation, 20 rounds, consensus distance every round."""
-    Scenario(16, 65536 + 12, ("hypercube", 0.1), ("hypercube", 0.1), seed=0, mode=mode).run(20)
+    Scenario(16, 65536 + 12, ("hypercube", 0.1), ("hypercube", 0.1), seed=0, mode=mode, path=path).run(20)
 
 
-def test_config5_reduced():
+@pytest.mark.parametrize("path", PATHS)
+def test_config5_reduced(path):
     """K=64 dense Sinkhorn Mix2, Mix1 mean, 5 rounds."""
-    Scenario(64, 40000, ("mean",), ("dense", SINK64), seed=0).run(5)
+    Scenario(64, 40000, ("mean",), ("dense", SINK64), seed=0, path=path).run(5)
 
 
 def test_pairwise_gossip_presets():
