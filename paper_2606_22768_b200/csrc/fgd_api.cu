@@ -215,64 +215,94 @@ int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc) {
   return FGD_OK;
 }
 
-constexpr int kConsumers = 128;  // consumer threads per CTA of the TMA kernel (+ one producer warp)
-
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Can the TMA kernel run this call?  Writes the vector width and stage count to use.
-bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, int* vec_out, int* stages_out) {
+// Tile shapes of the TMA kernel.  A stage holds n_tensors x K x (consumers * vec) floats and at
+// least two stages must fit in shared memory; measured on B200, 256 consumer threads with
+// K * vec = 32 (a 96 KB stage, two stages) is the fastest shape, narrower tiles are the
+// fall-back when the Mix1 result is a staged matrix (four tensors per stage).
+struct TmaShape {
+  int vec, consumers, stages;
+};
+const int kTmaShapes[][3] = {  // {KT, vec, consumers}, in order of preference per KT
+    {0, 1, 128},
+    {2, 4, 256}, {2, 4, 128},
+    {4, 4, 256}, {4, 4, 128},
+    {8, 4, 256}, {8, 4, 128},
+    {16, 2, 256}, {16, 2, 128},
+    {32, 1, 256}, {32, 1, 128},
+    {64, 1, 128},
+};
+
+size_t tma_fixed_smem(int K, int KT, bool dense2, int consumers) {
+  return 128 + (dense2 ? sizeof(float) * K * K : 0) + (KT == 0 ? sizeof(float) * K * consumers : 0);
+}
+
+// Can the TMA kernel run this call?  Picks the tile shape.
+bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* out) {
   if (!c->encode_tiled) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
   const int K = c->K, KT = kt_of(K), NT = a.xsrc == XSRC_MATRIX ? 4 : 3;
-  const size_t fixed = 128 + 4096 + (dense2 ? sizeof(float) * K * K : 0) + (KT == 0 ? sizeof(float) * K * kConsumers : 0);
-  for (int vec = want_vec(KT); vec >= 1; vec >>= 1) {
-    if (c->P % vec != 0) continue;
-    if (vec > 1 && a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
-    const size_t stage = tma_stage_bytes(K, kConsumers * vec, NT);
-    if ((size_t)c->max_smem_optin < fixed + 2 * stage) continue;
-    int stages = (int)(((size_t)c->max_smem_optin - fixed) / stage);
+  const size_t budget = (size_t)c->max_smem_optin - 4096;  // static shared memory + slack
+  for (const auto& sh : kTmaShapes) {
+    if (sh[0] != KT) continue;
+    const int vec = sh[1], consumers = sh[2];
+    if (a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
+    const size_t fixed = tma_fixed_smem(K, KT, dense2, consumers);
+    const size_t stage = tma_stage_bytes(K, consumers * vec, NT);
+    if (budget < fixed + 2 * stage) continue;
+    int stages = (int)((budget - fixed) / stage);
     if (stages > kMaxStages) stages = kMaxStages;
-    *vec_out = vec;
-    *stages_out = stages;
+    *out = {vec, consumers, stages};
     return true;
   }
   return false;
 }
 
 int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
-                    const GatherMix& g1, int vec, int stages, cudaStream_t st, int* grid_out) {
+                    const GatherMix& g1, TmaShape sh, cudaStream_t st, int* grid_out) {
   const int K = c->K, KT = kt_of(K);
   TmaStepArgs ta;
   ta.s = a;
   ta.status = c->status;
   ta.n_tensors = a.xsrc == XSRC_MATRIX ? 4 : 3;
-  ta.stages = stages;
-  const int T = kConsumers * vec;
+  ta.stages = sh.stages;
+  const int T = sh.consumers * sh.vec;
   const int boxc = T < 256 ? T : 256;
   CUtensorMap tp, tl, tm, tx;
   if (int rc = make_tensor_map(c, &tp, a.theta_prev, boxc)) return rc;
   if (int rc = make_tensor_map(c, &tl, a.theta_local, boxc)) return rc;
   if (int rc = make_tensor_map(c, &tm, a.momentum, boxc)) return rc;
   if (int rc = make_tensor_map(c, &tx, a.xsrc == XSRC_MATRIX ? a.x : a.theta_prev, boxc)) return rc;
-  const size_t smem = 128 + tma_stage_bytes(K, T, ta.n_tensors) * stages + (dense2 ? sizeof(float) * K * K : 0) +
-                      (KT == 0 ? sizeof(float) * K * kConsumers : 0);
+  const size_t smem = tma_fixed_smem(K, KT, dense2, sh.consumers) + tma_stage_bytes(K, T, ta.n_tensors) * sh.stages;
   const int64_t ntiles = (c->P + T - 1) / T;
-  return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
+  auto go = [&]<int KTc, int VECc, int Cc>() -> int {
     int grid = 0;
     if (dense2) {
-      auto kern = outer_step_tma_kernel<KTc, VECc, kConsumers, true, DenseMix>;
-      if (int r = persistent_grid(c, kern, kConsumers + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, kConsumers + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
+      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, true, DenseMix>;
+      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
+      kern<<<grid, Cc + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
     } else {
-      auto kern = outer_step_tma_kernel<KTc, VECc, kConsumers, false, GatherMix>;
-      if (int r = persistent_grid(c, kern, kConsumers + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, kConsumers + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
+      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, false, GatherMix>;
+      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
+      kern<<<grid, Cc + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
     }
     *grid_out = grid;
     return check_launch(c, "outer_step_tma_kernel");
-  });
+  };
+#define FGD_TMA_CASE(kt, v, cc) \
+  if (KT == kt && sh.vec == v && sh.consumers == cc) return go.template operator()<kt, v, cc>();
+  FGD_TMA_CASE(0, 1, 128)
+  FGD_TMA_CASE(2, 4, 256) FGD_TMA_CASE(2, 4, 128)
+  FGD_TMA_CASE(4, 4, 256) FGD_TMA_CASE(4, 4, 128)
+  FGD_TMA_CASE(8, 4, 256) FGD_TMA_CASE(8, 4, 128)
+  FGD_TMA_CASE(16, 2, 256) FGD_TMA_CASE(16, 2, 128)
+  FGD_TMA_CASE(32, 1, 256) FGD_TMA_CASE(32, 1, 128)
+  FGD_TMA_CASE(64, 1, 128)
+#undef FGD_TMA_CASE
+  return fail(c, FGD_ERR_UNSUPPORTED, "internal: no TMA kernel for this shape");
 }
 
 }  // namespace
@@ -477,13 +507,13 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
   const int KT = kt_of(K);
   int grid = 0;
   int rc = FGD_OK;
-  int tma_vec = 0, tma_stages = 0;
-  const bool can_tma = tma_eligible(c, a, dense2, &tma_vec, &tma_stages);
+  TmaShape shape{0, 0, 0};
+  const bool can_tma = tma_eligible(c, a, dense2, &shape);
   if (c->path == FGD_PATH_TMA && !can_tma)
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   if (can_tma && c->path != FGD_PATH_REGISTER) {
-    rc = launch_step_tma(c, a, dense2, g2, d2, g1, tma_vec, tma_stages, st, &grid);
+    rc = launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x});
     rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {

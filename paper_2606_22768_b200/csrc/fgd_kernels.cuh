@@ -90,24 +90,108 @@ struct SCol<1> {
   }
 };
 
+// ---- element-wise helpers on Pack<VEC>.  For even VEC they use the packed fp32x2
+// instructions of sm_100 (one issue slot for two lanes of the vector), which halves the
+// floating-point instruction count of these issue-bound streaming kernels.
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_fma(const Pack<VEC>& a, float s, const Pack<VEC>& c) {  // a*s + c
+  Pack<VEC> r;
+  if constexpr (VEC % 2 == 0) {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 2) {
+      const float2 t = __ffma2_rn(make_float2(a.v[i], a.v[i + 1]), make_float2(s, s), make_float2(c.v[i], c.v[i + 1]));
+      r.v[i] = t.x;
+      r.v[i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) r.v[i] = fmaf(a.v[i], s, c.v[i]);
+  }
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_fma(const Pack<VEC>& a, const Pack<VEC>& b, const Pack<VEC>& c) {  // a*b + c
+  Pack<VEC> r;
+  if constexpr (VEC % 2 == 0) {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 2) {
+      const float2 t = __ffma2_rn(make_float2(a.v[i], a.v[i + 1]), make_float2(b.v[i], b.v[i + 1]),
+                                  make_float2(c.v[i], c.v[i + 1]));
+      r.v[i] = t.x;
+      r.v[i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) r.v[i] = fmaf(a.v[i], b.v[i], c.v[i]);
+  }
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_add(const Pack<VEC>& a, const Pack<VEC>& b) {
+  Pack<VEC> r;
+  if constexpr (VEC % 2 == 0) {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 2) {
+      const float2 t = __fadd2_rn(make_float2(a.v[i], a.v[i + 1]), make_float2(b.v[i], b.v[i + 1]));
+      r.v[i] = t.x;
+      r.v[i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) r.v[i] = a.v[i] + b.v[i];
+  }
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_mul(const Pack<VEC>& a, float s) {
+  Pack<VEC> r;
+  if constexpr (VEC % 2 == 0) {
+#pragma unroll
+    for (int i = 0; i < VEC; i += 2) {
+      const float2 t = __fmul2_rn(make_float2(a.v[i], a.v[i + 1]), make_float2(s, s));
+      r.v[i] = t.x;
+      r.v[i + 1] = t.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) r.v[i] = a.v[i] * s;
+  }
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_sub(const Pack<VEC>& a, const Pack<VEC>& b) {  // a - b (exact: b * -1 + a)
+  return p_fma<VEC>(b, -1.0f, a);
+}
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> p_zero() {
+  Pack<VEC> r;
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) r.v[i] = 0.f;
+  return r;
+}
+template <int VEC>
+__device__ __forceinline__ float p_hsum(const Pack<VEC>& a) {
+  float s = a.v[0];
+#pragma unroll
+  for (int i = 1; i < VEC; ++i) s += a.v[i];
+  return s;
+}
+
 // Gather of a mix row from a thread-private shared column:
 //   out = w_self[m] * col[m] + sum_{j < D} w[m][j] * col[nbr[m][j]]
 template <int VEC, int BLOCK>
 __device__ __forceinline__ Pack<VEC> gather_row(const GatherMix& mx, int m, const float* col, int tid) {
   Pack<VEC> acc;
   const Pack<VEC> self = SCol<VEC>::ld(col, m * BLOCK + tid);
-  const float ws = mx.w_self[m];
-#pragma unroll
-  for (int i = 0; i < VEC; ++i) acc.v[i] = ws * self.v[i];
-#pragma unroll
-  for (int j = 0; j < FGD_MAX_D; ++j) {
-    if (j < mx.D) {
-      const int n = mx.nbr[m * FGD_MAX_D + j];
-      const float wj = mx.w[m * FGD_MAX_D + j];
-      const Pack<VEC> t = SCol<VEC>::ld(col, n * BLOCK + tid);
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) acc.v[i] = fmaf(wj, t.v[i], acc.v[i]);
-    }
+  acc = p_mul<VEC>(self, mx.w_self[m]);
+  // D is warp-uniform: a real loop issues D slots, where an unrolled predicated one would
+  // issue all FGD_MAX_D of them
+  const int D = mx.D;
+#pragma unroll 1
+  for (int j = 0; j < D; ++j) {
+    const int n = mx.nbr[m * FGD_MAX_D + j];
+    const float wj = mx.w[m * FGD_MAX_D + j];
+    acc = p_fma<VEC>(SCol<VEC>::ld(col, n * BLOCK + tid), wj, acc);
   }
   return acc;
 }

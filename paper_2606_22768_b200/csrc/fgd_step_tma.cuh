@@ -85,6 +85,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
   constexpr int NBOX = T / BOXC;              // boxes per tensor per tile
   constexpr int TPB = BOXC / VEC;             // consumer threads per box
   constexpr int NWARP = CONSUMERS / 32 + 1;
+  static_assert(T % BOXC == 0 && CONSUMERS % 32 == 0 && BOXC % VEC == 0, "tile must be whole TMA boxes");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * kMaxStages];
   __shared__ int abort_flag;
@@ -173,8 +174,14 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
       const uint32_t use = (uint32_t)(i / STAGES);
       const int64_t col = tile * T + (int64_t)tid * VEC;
       const bool live = col < P;
-      Pack<VEC> xv;
-      if (a.xsrc == XSRC_VECTOR && live) xv = ld_stream<VEC>(a.x + col);   // latency hides behind the wait
+      const bool whole = col + VEC <= P;       // false only for the one group that straddles P
+      Pack<VEC> xv = p_zero<VEC>();
+      if (a.xsrc == XSRC_VECTOR && live) {     // latency hides behind the wait
+        if (whole) xv = ld_stream<VEC>(a.x + col);
+        else
+          for (int q = 0; q < VEC; ++q)
+            if (col + q < P) xv.v[q] = a.x[col + q];
+      }
       if (!mbar_wait(smem_u32(&bars[s]), use & 1)) {
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
@@ -188,51 +195,77 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
       float* X = C + tens_floats;              // Mix1 result (matrix), if staged
       const int t = tid % TPB;
       if (live) {
+        // With a compile-time K every per-worker value has a static register index, so all
+        // shared-memory loads of a phase are issued before anything depends on them and
+        // theta_new never goes back to shared memory.  (Runtime K keeps them in the stage.)
+        constexpr bool REGS = (KT > 0) && !(DENSE2 && KT > 16);
+        constexpr int KQ = REGS ? KT : 1;
         // ---- phase 1: outer gradients of all workers into B, column sums
-        Pack<VEC> gsum, tsum;
+        Pack<VEC> gsum = p_zero<VEC>(), tsum = p_zero<VEC>();
+        const bool need_tsum = a.xsrc == XSRC_FUSED && m1.kind == KMIX_MEAN;
+        if constexpr (REGS) {
+          Pack<VEC> tpv[KQ], tlv[KQ];
 #pragma unroll
-        for (int q = 0; q < VEC; ++q) gsum.v[q] = tsum.v[q] = 0.f;
-#pragma unroll(KT > 0 ? KT : 4)
-        for (int m = 0; m < K; ++m) {
-          const Pack<VEC> tp = SCol<VEC>::ld(A, m * TPB + t);
-          const Pack<VEC> tl = SCol<VEC>::ld(B, m * TPB + t);
-          Pack<VEC> g;
-#pragma unroll
-          for (int q = 0; q < VEC; ++q) {
-            g.v[q] = tp.v[q] - tl.v[q];
-            gsum.v[q] += g.v[q];
-            tsum.v[q] += tp.v[q];
+          for (int m = 0; m < KQ; ++m) {
+            tpv[m] = SCol<VEC>::ld(A, m * TPB + t);
+            tlv[m] = SCol<VEC>::ld(B, m * TPB + t);
           }
-          SCol<VEC>::st(B, m * TPB + t, g);
-        }
-        if (a.xsrc != XSRC_VECTOR) {
 #pragma unroll
-          for (int q = 0; q < VEC; ++q) xv.v[q] = tsum.v[q] * invK;   // fused mean Mix1
-        }
-        Pack<VEC> gmean, asum;
+          for (int m = 0; m < KQ; ++m) {
+            const Pack<VEC> g = p_sub<VEC>(tpv[m], tlv[m]);
+            gsum = p_add<VEC>(gsum, g);
+            SCol<VEC>::st(B, m * TPB + t, g);
+          }
+          if (need_tsum) {
 #pragma unroll
-        for (int q = 0; q < VEC; ++q) {
-          gmean.v[q] = gsum.v[q] * invK;
-          asum.v[q] = 0.f;
+            for (int m = 0; m < KQ; ++m) tsum = p_add<VEC>(tsum, tpv[m]);
+          }
+        } else {
+#pragma unroll 4
+          for (int m = 0; m < K; ++m) {
+            const Pack<VEC> tp = SCol<VEC>::ld(A, m * TPB + t);
+            const Pack<VEC> tl = SCol<VEC>::ld(B, m * TPB + t);
+            const Pack<VEC> g = p_sub<VEC>(tp, tl);
+            gsum = p_add<VEC>(gsum, g);
+            tsum = p_add<VEC>(tsum, tp);
+            SCol<VEC>::st(B, m * TPB + t, g);
+          }
         }
-        // ---- phase 2: mix, Nesterov step, stream out, keep theta_new in C
+        if (a.xsrc != XSRC_VECTOR) xv = p_mul<VEC>(tsum, invK);   // fused mean Mix1
+        const Pack<VEC> gmean = p_mul<VEC>(gsum, invK);
+        Pack<VEC> asum = p_zero<VEC>();
+        // ---- phase 2: mix, Nesterov step, stream out; theta_new stays in av[] (or in C)
+        Pack<VEC> av[KQ];
+        if constexpr (REGS) {
+#pragma unroll
+          for (int m = 0; m < KQ; ++m) av[m] = SCol<VEC>::ld(C, m * TPB + t);   // momentum, all rows
+        }
+        float* const mom_col = a.momentum + col;
+        float* const new_col = a.theta_new + col;
         auto finish_row = [&](int m, const Pack<VEC>& gh) {
-          const size_t off = (size_t)m * ld + col;
+          const size_t off = (size_t)m * ld;
           Pack<VEC> xm;
           if (a.xsrc == XSRC_MATRIX) xm = SCol<VEC>::ld(X, m * TPB + t);
           else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) xm = gather_row<VEC, TPB>(m1, m, A, t);
           else xm = xv;
-          const Pack<VEC> v = SCol<VEC>::ld(C, m * TPB + t);
-          Pack<VEC> vn, tn;
-#pragma unroll
-          for (int q = 0; q < VEC; ++q) {
-            vn.v[q] = fmaf(mu, v.v[q], gh.v[q]);
-            tn.v[q] = xm.v[q] - lr * fmaf(mu, vn.v[q], gh.v[q]);
-            asum.v[q] += tn.v[q];
+          Pack<VEC> v;
+          if constexpr (REGS) v = av[m];
+          else v = SCol<VEC>::ld(C, m * TPB + t);
+          const Pack<VEC> vn = p_fma<VEC>(v, mu, gh);                       // v' = mu v + ghat
+          const Pack<VEC> tn = p_fma<VEC>(p_fma<VEC>(vn, mu, gh), -lr, xm);   // x - lr (ghat + mu v')
+          asum = p_add<VEC>(asum, tn);
+          if (whole) {
+            st_stream<VEC>(mom_col + off, vn);
+            st_stream<VEC>(new_col + off, tn);
+          } else {                              // columns at or beyond P exist only as zero fill
+            for (int q = 0; q < VEC; ++q)
+              if (col + q < P) {
+                mom_col[off + q] = vn.v[q];
+                new_col[off + q] = tn.v[q];
+              }
           }
-          st_stream<VEC>(a.momentum + off, vn);
-          st_stream<VEC>(a.theta_new + off, tn);
-          if (want_cd) SCol<VEC>::st(C, m * TPB + t, tn);
+          if constexpr (REGS) av[m] = tn;
+          else if (want_cd) SCol<VEC>::st(C, m * TPB + t, tn);
         };
         if constexpr (DENSE2) {
           dense_rows<KT, VEC, TPB, (KT > 0 && KT <= 16)>(K, wts, B, t, finish_row);
@@ -247,15 +280,19 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
         }
         // ---- phase 3: squared deviation of theta_new from its column mean
         if (want_cd) {
+          const Pack<VEC> nmean = p_mul<VEC>(asum, -invK);
 #pragma unroll(KT > 0 ? KT : 4)
           for (int m = 0; m < K; ++m) {
-            const Pack<VEC> tv = SCol<VEC>::ld(C, m * TPB + t);
-            float sq = 0.f;
+            Pack<VEC> tv;
+            if constexpr (REGS) tv = av[m];
+            else tv = SCol<VEC>::ld(C, m * TPB + t);
+            Pack<VEC> d = p_add<VEC>(tv, nmean);
+            if (!whole) {
 #pragma unroll
-            for (int q = 0; q < VEC; ++q) {
-              const float d = tv.v[q] - asum.v[q] * invK;
-              sq = fmaf(d, d, sq);
+              for (int q = 0; q < VEC; ++q)
+                if (col + q >= P) d.v[q] = 0.f;
             }
+            const float sq = p_hsum<VEC>(p_fma<VEC>(d, d, p_zero<VEC>()));
             if constexpr (KT > 0) sacc[m] += sq;
             else sas[m * CONSUMERS + tid] += sq;
           }
