@@ -154,6 +154,23 @@ int fgd_outer_step(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* m
  * fgd_cd_finalize. */
 int fgd_consensus_distance(fgd_ctx* ctx, const float* theta, double* cd_sumsq, void* stream);
 
+/* (No counterpart in the paper: a packaging variant of fgd_consensus_distance.)
+ * Same result as fgd_consensus_distance, for callers that cannot allocate GPU memory and so
+ * cannot create a context: it needs no fgd_ctx and calls no cudaMalloc / cudaFree or any other
+ * allocating routine.  Its per-CTA partial sums live in a fixed 512 KiB device array that is
+ * part of the library image (1024 CTAs x FGD_MAX_K workers x 8 bytes), resident on every GPU
+ * that loads the library until the process exits.
+ *   device, K, P, ld   as in fgd_create; K > FGD_MAX_K does not fit the array and is rejected
+ *                      with FGD_ERR_INVALID_ARG (any P is fine: the grid is capped at 1024 CTAs).
+ *   theta              device [K, ld] fp32; cd_sumsq device [K] doubles (caller-owned).
+ * The first call on a device resolves the array's device address (once per device); make that
+ * first call before starting any stream capture.  All calls share the one array and it keeps
+ * the previous call's contents (nothing in it needs to start at zero): two calls that overlap
+ * on the same GPU race and return wrong sums, so order them on one stream or with events.
+ * Errors: reason via fgd_last_error(NULL). */
+int fgd_consensus_distance_noalloc(int device, int K, int64_t P, int64_t ld, const float* theta,
+                                   double* cd_sumsq, void* stream);
+
 /* ---------------------------- host helpers (pure CPU) ---------------------------------- */
 /* Topologies.  Each writes nbr[K*D], w[K*D], w_self[K] for the D it documents and returns D
  * (>= 0) or a negative status.  Weights are Metropolis weights of the unmasked graph.

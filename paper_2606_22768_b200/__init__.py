@@ -52,7 +52,7 @@ class _CMixDesc(ctypes.Structure):
 
 def _load():
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2606_22768_b200.build` "
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python paper_2606_22768_b200/build.py` "
                           "(there is no CPU fallback)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, i64, u64, dbl = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_double
@@ -69,6 +69,7 @@ def _load():
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
         "fgd_consensus_distance": (i32, [vp, vp, vp, vp]),
+        "fgd_consensus_distance_noalloc": (i32, [i32, i32, i64, i64, vp, vp, vp]),
         "fgd_topo_ring": (i32, [i32, vp, vp, vp]),
         "fgd_topo_onepeer_xor": (i32, [i32, i64, vp, vp, vp]),
         "fgd_topo_hypercube": (i32, [i32, vp, vp, vp]),
@@ -304,3 +305,14 @@ def fgd_outer_step(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x
 def fgd_consensus_distance(ctx: Context, theta, cd_sumsq, stream=None) -> None:
     ctx._check(_lib.fgd_consensus_distance(ctx._h, _dev_ptr(theta, "theta", "torch.float32"),
                                            _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), _stream(stream)))
+
+
+def fgd_consensus_distance_noalloc(device: int, K: int, P: int, ld: int, theta, cd_sumsq, stream=None) -> None:
+    """Consensus sums without a context and without any GPU allocation (for callers that may not
+    allocate); partial sums go through a fixed array inside the library, shared by all calls, so
+    calls on one GPU must not overlap.  See ``include/fgd.h``."""
+    rc = _lib.fgd_consensus_distance_noalloc(int(device), int(K), int(P), int(ld),
+                                             _dev_ptr(theta, "theta", "torch.float32"),
+                                             _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), _stream(stream))
+    if rc != 0:
+        raise FgdError(rc, fgd_last_error(None))

@@ -1,6 +1,7 @@
 """Build ``libfgd.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-Run as ``python -m paper_2606_22768_b200.build``.  Needs only nvcc (cross-compiles without
+Run as ``python paper_2606_22768_b200/build.py`` (as a script: importing the package needs the
+library to exist already).  Needs only nvcc (cross-compiles without
 a GPU).  The library links the CUDA runtime statically, so it loads on machines without a
 driver; only the GPU entry points then fail (with FGD_ERR_CUDA).
 """
@@ -14,8 +15,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfgd.so")
-SOURCES = ["fgd_api.cu", "fgd_host.cpp"]
-HEADERS = ["fgd_kernels.cuh", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
+SOURCES = ["fgd_api.cu", "fgd_noalloc.cu", "fgd_host.cpp"]
+HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
 
 NVCC_FLAGS = ["-std=c++20", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-I" + os.path.join(ROOT, "include")]

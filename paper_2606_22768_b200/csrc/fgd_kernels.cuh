@@ -583,7 +583,7 @@ consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials,
 
 // out[m] = sum_b partials[b][m], fixed order: one warp per worker, lanes stride the blocks,
 // then a shuffle tree.  Deterministic.
-__global__ void __launch_bounds__(32)
+static __global__ void __launch_bounds__(32)
 consensus_finalize_kernel(const double* __restrict__ partials, int nblocks, int K, double* __restrict__ out) {
   const int m = blockIdx.x, lane = threadIdx.x;
   double d = 0.0;
