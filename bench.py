@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS))
+    ap.add_argument("--cols", type=int, default=0,
+                    help="profiling only: shrink P to this many columns (same kernels, smaller launch)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -192,6 +194,20 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------- N > 1: replicas
+def aggregate(dist, elapsed_ms: float, units: int, device=None):
+    """Whole-job figures of N independent replicas: the slowest rank's time and the sum of the
+    units all ranks processed.  `dist` is torch.distributed (any backend) or None for N = 1."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return elapsed_ms, units
+    import torch
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(u.item())
+
+
 # ---------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -211,7 +227,10 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = CONFIGS[args.config]
+    cfg = dict(CONFIGS[args.config])
+    if args.cols:
+        cfg["P"] = args.cols
+        cfg["name"] += f" [REDUCED to P={args.cols} for profiling: not a benchmark number]"
     K, P, seed = cfg["K"], cfg["P"], 0
     steps, warmup = args.steps, max(args.warmup, 3)
     sig = gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1] else np.full(K, cfg["sig"][0], np.float32)
@@ -259,13 +278,10 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     if world > 1:
         dist.barrier()
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms, units = aggregate(dist if world > 1 else None, elapsed_ms, K * P, dev)
     kern_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs)
 
     ms_per_step = elapsed_ms / steps
-    units = K * P * world
     value = units / (ms_per_step * 1e-3)
     x_vec = cfg["mix1"][0] == "mean"
     step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
@@ -274,7 +290,7 @@ def run_ours(args):
     achieved = step_bytes / (kern_ms * 1e-3) / 1e9
     tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if tr is None else tr * K * P, "kernel": "outer_step_kernel",
+                "traffic": None if tr is None else tr * K * P, "kernel": "outer_step_tma_kernel",
                 "kernel_ms": kern_ms, "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / 8000.0}
 
@@ -373,11 +389,8 @@ def e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W
     b.record(main)
     torch.cuda.synchronize()
     ms = a.elapsed_time(b)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return {"value": K * P * world / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": K * P * 4,
+    ms, units = aggregate(dist if world > 1 else None, ms, K * P, dev)
+    return {"value": units / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": K * P * 4,
             "d2h_bytes_per_step": K * 8, "steps": steps, "ms_per_step": ms / steps}
 
 

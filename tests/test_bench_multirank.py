@@ -1,0 +1,51 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks, whole-job time = slowest rank, units = sum."""
+import os
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms, units = bench.aggregate(dist, 10.0 + 5.0 * rank, 1000 * (rank + 1))
+    dist.barrier()
+    dist.destroy_process_group()
+    q.put((rank, ms, units))
+
+
+def test_aggregate_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + (os.getpid() % 2000)
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == [(0, 15.0, 3000), (1, 15.0, 3000)]
+
+
+def test_aggregate_single_process_is_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.aggregate(None, 12.5, 77) == (12.5, 77)
+
+
+def test_reference_arm_runs_on_rank0_only(monkeypatch, capsys):
+    """--impl reference under torchrun: ranks other than 0 print nothing and return."""
+    sys.path.insert(0, ROOT)
+    import bench
+    monkeypatch.setenv("RANK", "1")
+    args = type("A", (), dict(config=1, steps=1, warmup=0, gpus=2))()
+    bench.run_reference(args)
+    assert capsys.readouterr().out == ""
