@@ -51,7 +51,7 @@ CONFIGS = {
 # DRAM bytes per worker-parameter of the fused outer-step kernel measured with ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch / (K*P) of that launch); the
 # capture it comes from is summarised under profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: None}
+NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: 20.04}  # profiles/outer_step_tma_kernel_cfg3_16Mcols_ncu.md
 
 
 def parse_args():
@@ -279,7 +279,8 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     elapsed_ms, units = aggregate(dist if world > 1 else None, elapsed_ms, K * P, dev)
-    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs)
+    kern_times = [a.elapsed_time(b) for a, b in pairs]
+    kern_ms = statistics.mean(kern_times)
 
     ms_per_step = elapsed_ms / steps
     value = units / (ms_per_step * 1e-3)
@@ -291,7 +292,8 @@ def run_ours(args):
     tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if tr is None else tr * K * P, "kernel": "outer_step_tma_kernel",
-                "kernel_ms": kern_ms, "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
+                "kernel_ms": kern_ms, "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
+                "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / 8000.0}
 
     # consensus distance of the last round (both of the paper's definitions)
@@ -308,6 +310,9 @@ def run_ours(args):
             "roofline": roofline, "gpu_launches": int(launches), "clocks": clocks,
             "consensus": {"cd_norm": cd_norm, "cd_sq": cd_sq}}
 
+    if rank == 0:
+        # context: the same STREAM-style copy the pool's peak was measured with, on THIS box, now
+        roofline["copy_gbs_this_box"] = copy_bandwidth(torch, dev)
     if rank == 0 and not args.no_overlap:
         line["overlap"] = overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, dense_W)
     if not args.no_e2e:
@@ -319,6 +324,25 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def copy_bandwidth(torch, dev, n=1 << 30, reps=10):
+    """torch b.copy_(a) over 2^30 bf16 elements, read + write bytes, best of `reps` (GB/s)."""
+    try:
+        a = torch.empty(n, dtype=torch.bfloat16, device=dev)
+        b = torch.empty_like(a)
+    except Exception:
+        return None
+    best = None
+    for _ in range(reps + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        best = ms if best is None else min(best, ms)
+    return 2 * n * 2 / (best * 1e-3) / 1e9
 
 
 def overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, dense_W, reps=3):
