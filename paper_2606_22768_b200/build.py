@@ -15,11 +15,12 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfgd.so")
-SOURCES = ["fgd_api.cu", "fgd_noalloc.cu", "fgd_host.cpp"]
-HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
+SOURCES = ["fgd_api.cu", "fgd_step_tma.cu", "fgd_noalloc.cu", "fgd_host.cpp"]
+HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_step_tma.h", "fgd_ctx.h", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
 
 NVCC_FLAGS = ["-std=c++20", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-              "-Xcompiler", "-fPIC", "-shared", "-I" + os.path.join(ROOT, "include")]
+              "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include")]
+OBJ_DIR = os.path.join(HERE, "build")
 
 
 def stale() -> bool:
@@ -32,9 +33,18 @@ def stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or stale():
-        cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", OUT] + \
-              [os.path.join(CSRC, s) for s in SOURCES]
-        subprocess.run(cmd, check=True)
+        from concurrent.futures import ThreadPoolExecutor
+        os.makedirs(OBJ_DIR, exist_ok=True)
+        extra = ["-Xptxas", "-v"] if verbose else []
+
+        def compile_one(src):
+            obj = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + ".o")
+            subprocess.run(["nvcc"] + NVCC_FLAGS + extra + ["-c", "-o", obj, os.path.join(CSRC, src)], check=True)
+            return obj
+
+        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:   # one nvcc per translation unit
+            objs = list(pool.map(compile_one, SOURCES))
+        subprocess.run(["nvcc", "-shared", "-o", OUT] + objs, check=True)
     return OUT
 
 

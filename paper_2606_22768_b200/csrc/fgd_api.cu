@@ -6,303 +6,17 @@
 #include <map>
 #include <utility>
 
+#include "fgd_ctx.h"
 #include "fgd_kernels.cuh"
-#include "fgd_step_tma.cuh"
+#include "fgd_step_tma.h"
 
 using namespace fgd;
 
 namespace {
-constexpr int kBlock = 128;           // threads per CTA for the column kernels
-constexpr int kGradBlock = 256;
-constexpr int kMaxPartialBlocks = 148 * 16 * 2;
-}  // namespace
-
-struct fgd_ctx {
-  int device = 0;
-  int K = 0;
-  int64_t P = 0, ld = 0;
-  int num_sms = 0;
-  double* partials = nullptr;  // [kMaxPartialBlocks][K]
-  int* status = nullptr;       // device status word written by bounded waits that gave up
-  int path = FGD_PATH_AUTO;    // which fused-step kernel family to use
-  int max_smem_optin = 0;
-  void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
-  int64_t launches = 0;
-  char err[256] = "";
-  std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
-};
-
-namespace {
-
-int fail(fgd_ctx* c, int status, const char* fmt, ...) {
-  va_list ap;
-  va_start(ap, fmt);
-  if (c) vsnprintf(c->err, sizeof(c->err), fmt, ap);
-  else vsnprintf(g_thread_error, sizeof(g_thread_error), fmt, ap);
-  va_end(ap);
-  return status;
-}
-
-int cuda_fail(fgd_ctx* c, cudaError_t e, const char* what) {
-  return fail(c, FGD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
-}
-
-#define FGD_CUDA(c, call)                                   \
-  do {                                                      \
-    cudaError_t e_ = (call);                                \
-    if (e_ != cudaSuccess) return cuda_fail(c, e_, #call);  \
-  } while (0)
-
-// Byte range a [K, ld] matrix with P used columns occupies.
-struct Range {
-  uintptr_t lo, hi;
-};
-Range mat_range(const void* p, int K, int64_t P, int64_t ld) {
-  const uintptr_t b = reinterpret_cast<uintptr_t>(p);
-  return {b, b + (uintptr_t)(((int64_t)(K - 1) * ld + P) * (int64_t)sizeof(float))};
-}
-Range vec_range(const void* p, int64_t n, size_t elt) {
-  const uintptr_t b = reinterpret_cast<uintptr_t>(p);
-  return {b, b + (uintptr_t)n * elt};
-}
-bool overlap(Range a, Range b) { return a.lo < b.hi && b.lo < a.hi; }
-
-// Widest vector width usable for these pointers / sizes, capped at `want`.
-int pick_vec(int want, int64_t P, int64_t ld, std::initializer_list<const void*> ptrs) {
-  for (int v = want; v > 1; v >>= 1) {
-    bool ok = (P % v == 0) && (ld % v == 0);
-    for (const void* p : ptrs)
-      if (p && (reinterpret_cast<uintptr_t>(p) % (sizeof(float) * v)) != 0) ok = false;
-    if (ok) return v;
-  }
-  return 1;
-}
-
-// Kernel-side description of a non-dense mix (identity / mean / sparse).
-int make_gather(fgd_ctx* c, const fgd_mix_desc* d, GatherMix* out) {
-  const int K = d->K;
-  memset(out, 0, sizeof(*out));
-  if (d->kind == FGD_MIX_MEAN) {
-    out->kind = KMIX_MEAN;
-    return FGD_OK;
-  }
-  out->kind = KMIX_GATHER;
-  for (int m = 0; m < K; ++m) {
-    out->w_self[m] = 1.f;
-    for (int j = 0; j < FGD_MAX_D; ++j) out->nbr[m * FGD_MAX_D + j] = m;
-  }
-  if (d->kind == FGD_MIX_IDENTITY) return FGD_OK;
-  if (d->kind != FGD_MIX_SPARSE) return fail(c, FGD_ERR_INVALID_ARG, "internal: not a gather mix");
-  double w_eff[FGD_MAX_K * FGD_MAX_D], ws_eff[FGD_MAX_K];
-  effective_weights(d, w_eff, ws_eff);
-  out->D = d->D;
-  for (int m = 0; m < K; ++m) {
-    out->w_self[m] = (float)ws_eff[m];
-    for (int j = 0; j < d->D; ++j) {
-      const int n = d->nbr[m * d->D + j];
-      out->nbr[m * FGD_MAX_D + j] = n >= 0 ? n : m;
-      out->w[m * FGD_MAX_D + j] = n >= 0 ? (float)w_eff[m * d->D + j] : 0.f;
-    }
-  }
-  return FGD_OK;
-}
-
-void make_dense(const fgd_mix_desc* d, DenseMix* out) {
-  const int K = d->K;
-  for (int m = 0; m < K; ++m)
-    for (int n = 0; n < K; ++n) out->Wt[n * K + m] = d->W[m * K + n];
-}
-
-// CTAs per SM for (kernel, block, smem); raises the dynamic shared-memory limit when needed.
-template <typename Kern>
-int ctas_per_sm(fgd_ctx* c, Kern kern, int block, size_t smem, int* out) {
-  const auto key = std::make_pair(reinterpret_cast<const void*>(kern), smem);
-  auto it = c->occupancy.find(key);
-  if (it != c->occupancy.end()) {
-    *out = it->second;
-    return FGD_OK;
-  }
-  if (smem > 48 * 1024)
-    FGD_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  int n = 0;
-  FGD_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, block, smem));
-  if (n < 1) return fail(c, FGD_ERR_UNSUPPORTED, "kernel does not fit on an SM (smem %zu B)", smem);
-  c->occupancy[key] = n;
-  *out = n;
-  return FGD_OK;
-}
-
-template <typename Kern>
-int persistent_grid(fgd_ctx* c, Kern kern, int block, size_t smem, int64_t ntiles, int* grid) {
-  int per_sm = 0;
-  if (int rc = ctas_per_sm(c, kern, block, smem, &per_sm)) return rc;
-  int64_t g = (int64_t)per_sm * c->num_sms;
-  if (g > ntiles) g = ntiles;
-  if (g > kMaxPartialBlocks) g = kMaxPartialBlocks;
-  if (g < 1) g = 1;
-  *grid = (int)g;
-  return FGD_OK;
-}
-
-int check_launch(fgd_ctx* c, const char* what) {
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(c, e, what);
-  c->launches += 1;
-  return FGD_OK;
-}
-
-struct DeviceGuard {
-  int prev = -1;
-  bool ok = true;
-  explicit DeviceGuard(int dev) {
-    if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
-    else if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-  }
-  ~DeviceGuard() {
-    if (prev >= 0) cudaSetDevice(prev);
-  }
-};
-
-// ---- compile-time K / vector width selection -------------------------------------------
-// KT = K for the instantiated worker counts, 0 (runtime-K generic kernel) otherwise.
-int kt_of(int K) {
-  switch (K) {
-    case 2: case 4: case 8: case 16: case 32: case 64: return K;
-    default: return 0;
-  }
-}
-int want_vec(int KT) { return KT == 0 ? 1 : (KT <= 16 ? 4 : (KT == 32 ? 2 : 1)); }
-
-// Calls f.template operator()<KT, VEC>() for the (KT, VEC) pair chosen at run time.
-template <typename F>
-int dispatch_kv(int KT, int VEC, F&& f) {
-#define FGD_CASE(kt, v) \
-  if (KT == kt && VEC == v) return f.template operator()<kt, v>();
-  FGD_CASE(0, 1)
-  FGD_CASE(2, 4) FGD_CASE(2, 2) FGD_CASE(2, 1)
-  FGD_CASE(4, 4) FGD_CASE(4, 2) FGD_CASE(4, 1)
-  FGD_CASE(8, 4) FGD_CASE(8, 2) FGD_CASE(8, 1)
-  FGD_CASE(16, 4) FGD_CASE(16, 2) FGD_CASE(16, 1)
-  FGD_CASE(32, 2) FGD_CASE(32, 1)
-  FGD_CASE(64, 1)
-#undef FGD_CASE
-  return FGD_ERR_UNSUPPORTED;
-}
 
 int launch_finalize(fgd_ctx* c, int nblocks, double* out, cudaStream_t st) {
   consensus_finalize_kernel<<<c->K, 32, 0, st>>>(c->partials, nblocks, c->K, out);
   return check_launch(c, "consensus_finalize_kernel");
-}
-
-
-// ---- TMA-pipelined fused step ------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// 2-D map of a [K, ld] fp32 matrix restricted to its first P columns; box = boxc columns x K rows.
-// Columns at or beyond P read as zero.
-int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc) {
-  const cuuint64_t dims[2] = {(cuuint64_t)c->P, (cuuint64_t)c->K};
-  const cuuint64_t strides[1] = {(cuuint64_t)c->ld * sizeof(float)};
-  const cuuint32_t box[2] = {(cuuint32_t)boxc, (cuuint32_t)c->K};
-  const cuuint32_t estr[2] = {1, 1};
-  CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(
-      map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return fail(c, FGD_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
-  return FGD_OK;
-}
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-// Tile shapes of the TMA kernel.  A stage holds n_tensors x K x (consumers * vec) floats and at
-// least two stages must fit in shared memory; measured on B200, 256 consumer threads with
-// K * vec = 32 (a 96 KB stage, two stages) is the fastest shape, narrower tiles are the
-// fall-back when the Mix1 result is a staged matrix (four tensors per stage).
-struct TmaShape {
-  int vec, consumers, stages;
-};
-const int kTmaShapes[][3] = {  // {KT, vec, consumers}, in order of preference per KT
-    {0, 1, 128},
-    {2, 4, 256}, {2, 4, 128},
-    {4, 4, 256}, {4, 4, 128},
-    {8, 4, 256}, {8, 4, 128},
-    {16, 2, 256}, {16, 2, 128},
-    {32, 1, 256}, {32, 1, 128},
-    {64, 1, 128},
-};
-
-size_t tma_fixed_smem(int K, int KT, bool dense2, int consumers) {
-  return 128 + (dense2 ? sizeof(float) * K * K : 0) + (KT == 0 ? sizeof(float) * K * consumers : 0);
-}
-
-// Can the TMA kernel run this call?  Picks the tile shape.
-bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* out) {
-  if (!c->encode_tiled) return false;
-  if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
-  if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
-  if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
-  const int K = c->K, KT = kt_of(K), NT = a.xsrc == XSRC_MATRIX ? 4 : 3;
-  const size_t budget = (size_t)c->max_smem_optin - 4096;  // static shared memory + slack
-  for (const auto& sh : kTmaShapes) {
-    if (sh[0] != KT) continue;
-    const int vec = sh[1], consumers = sh[2];
-    if (a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
-    const size_t fixed = tma_fixed_smem(K, KT, dense2, consumers);
-    const size_t stage = tma_stage_bytes(K, consumers * vec, NT);
-    if (budget < fixed + 2 * stage) continue;
-    int stages = (int)((budget - fixed) / stage);
-    if (stages > kMaxStages) stages = kMaxStages;
-    *out = {vec, consumers, stages};
-    return true;
-  }
-  return false;
-}
-
-int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
-                    const GatherMix& g1, TmaShape sh, cudaStream_t st, int* grid_out) {
-  const int K = c->K, KT = kt_of(K);
-  TmaStepArgs ta;
-  ta.s = a;
-  ta.status = c->status;
-  ta.n_tensors = a.xsrc == XSRC_MATRIX ? 4 : 3;
-  ta.stages = sh.stages;
-  const int T = sh.consumers * sh.vec;
-  const int boxc = T < 256 ? T : 256;
-  CUtensorMap tp, tl, tm, tx;
-  if (int rc = make_tensor_map(c, &tp, a.theta_prev, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tl, a.theta_local, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tm, a.momentum, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tx, a.xsrc == XSRC_MATRIX ? a.x : a.theta_prev, boxc)) return rc;
-  const size_t smem = tma_fixed_smem(K, KT, dense2, sh.consumers) + tma_stage_bytes(K, T, ta.n_tensors) * sh.stages;
-  const int64_t ntiles = (c->P + T - 1) / T;
-  auto go = [&]<int KTc, int VECc, int Cc>() -> int {
-    int grid = 0;
-    if (dense2) {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, true, DenseMix>;
-      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, Cc + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
-    } else {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, false, GatherMix>;
-      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, Cc + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
-    }
-    *grid_out = grid;
-    return check_launch(c, "outer_step_tma_kernel");
-  };
-#define FGD_TMA_CASE(kt, v, cc) \
-  if (KT == kt && sh.vec == v && sh.consumers == cc) return go.template operator()<kt, v, cc>();
-  FGD_TMA_CASE(0, 1, 128)
-  FGD_TMA_CASE(2, 4, 256) FGD_TMA_CASE(2, 4, 128)
-  FGD_TMA_CASE(4, 4, 256) FGD_TMA_CASE(4, 4, 128)
-  FGD_TMA_CASE(8, 4, 256) FGD_TMA_CASE(8, 4, 128)
-  FGD_TMA_CASE(16, 2, 256) FGD_TMA_CASE(16, 2, 128)
-  FGD_TMA_CASE(32, 1, 256) FGD_TMA_CASE(32, 1, 128)
-  FGD_TMA_CASE(64, 1, 128)
-#undef FGD_TMA_CASE
-  return fail(c, FGD_ERR_UNSUPPORTED, "internal: no TMA kernel for this shape");
 }
 
 }  // namespace
@@ -507,13 +221,13 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
   const int KT = kt_of(K);
   int grid = 0;
   int rc = FGD_OK;
-  TmaShape shape{0, 0, 0};
-  const bool can_tma = tma_eligible(c, a, dense2, &shape);
+  FgdTmaShape shape{0, 0, 0};
+  const bool can_tma = fgd_tma_eligible(c, a, dense2, &shape);
   if (c->path == FGD_PATH_TMA && !can_tma)
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   if (can_tma && c->path != FGD_PATH_REGISTER) {
-    rc = launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
+    rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x});
     rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {

@@ -1,0 +1,198 @@
+// Context structure and small host helpers shared by the translation units that launch kernels.
+#ifndef FGD_CTX_H_
+#define FGD_CTX_H_
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <initializer_list>
+#include <map>
+#include <utility>
+
+#include "fgd_internal.h"
+
+using namespace fgd;  // internal header: only included by this library's own translation units
+
+namespace {
+constexpr int kBlock = 128;           // threads per CTA for the column kernels
+constexpr int kGradBlock = 256;
+constexpr int kMaxPartialBlocks = 148 * 16 * 2;
+}  // namespace
+
+struct fgd_ctx {
+  int device = 0;
+  int K = 0;
+  int64_t P = 0, ld = 0;
+  int num_sms = 0;
+  double* partials = nullptr;  // [kMaxPartialBlocks][K]
+  int* status = nullptr;       // device status word written by bounded waits that gave up
+  int path = FGD_PATH_AUTO;    // which fused-step kernel family to use
+  int max_smem_optin = 0;
+  void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
+  int64_t launches = 0;
+  char err[256] = "";
+  std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
+};
+
+namespace {
+
+int fail(fgd_ctx* c, int status, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  if (c) vsnprintf(c->err, sizeof(c->err), fmt, ap);
+  else vsnprintf(g_thread_error, sizeof(g_thread_error), fmt, ap);
+  va_end(ap);
+  return status;
+}
+
+int cuda_fail(fgd_ctx* c, cudaError_t e, const char* what) {
+  return fail(c, FGD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define FGD_CUDA(c, call)                                   \
+  do {                                                      \
+    cudaError_t e_ = (call);                                \
+    if (e_ != cudaSuccess) return cuda_fail(c, e_, #call);  \
+  } while (0)
+
+// Byte range a [K, ld] matrix with P used columns occupies.
+struct Range {
+  uintptr_t lo, hi;
+};
+Range mat_range(const void* p, int K, int64_t P, int64_t ld) {
+  const uintptr_t b = reinterpret_cast<uintptr_t>(p);
+  return {b, b + (uintptr_t)(((int64_t)(K - 1) * ld + P) * (int64_t)sizeof(float))};
+}
+Range vec_range(const void* p, int64_t n, size_t elt) {
+  const uintptr_t b = reinterpret_cast<uintptr_t>(p);
+  return {b, b + (uintptr_t)n * elt};
+}
+bool overlap(Range a, Range b) { return a.lo < b.hi && b.lo < a.hi; }
+
+// Widest vector width usable for these pointers / sizes, capped at `want`.
+int pick_vec(int want, int64_t P, int64_t ld, std::initializer_list<const void*> ptrs) {
+  for (int v = want; v > 1; v >>= 1) {
+    bool ok = (P % v == 0) && (ld % v == 0);
+    for (const void* p : ptrs)
+      if (p && (reinterpret_cast<uintptr_t>(p) % (sizeof(float) * v)) != 0) ok = false;
+    if (ok) return v;
+  }
+  return 1;
+}
+
+// Kernel-side description of a non-dense mix (identity / mean / sparse).
+int make_gather(fgd_ctx* c, const fgd_mix_desc* d, GatherMix* out) {
+  const int K = d->K;
+  memset(out, 0, sizeof(*out));
+  if (d->kind == FGD_MIX_MEAN) {
+    out->kind = KMIX_MEAN;
+    return FGD_OK;
+  }
+  out->kind = KMIX_GATHER;
+  for (int m = 0; m < K; ++m) {
+    out->w_self[m] = 1.f;
+    for (int j = 0; j < FGD_MAX_D; ++j) out->nbr[m * FGD_MAX_D + j] = m;
+  }
+  if (d->kind == FGD_MIX_IDENTITY) return FGD_OK;
+  if (d->kind != FGD_MIX_SPARSE) return fail(c, FGD_ERR_INVALID_ARG, "internal: not a gather mix");
+  double w_eff[FGD_MAX_K * FGD_MAX_D], ws_eff[FGD_MAX_K];
+  effective_weights(d, w_eff, ws_eff);
+  out->D = d->D;
+  for (int m = 0; m < K; ++m) {
+    out->w_self[m] = (float)ws_eff[m];
+    for (int j = 0; j < d->D; ++j) {
+      const int n = d->nbr[m * d->D + j];
+      out->nbr[m * FGD_MAX_D + j] = n >= 0 ? n : m;
+      out->w[m * FGD_MAX_D + j] = n >= 0 ? (float)w_eff[m * d->D + j] : 0.f;
+    }
+  }
+  return FGD_OK;
+}
+
+void make_dense(const fgd_mix_desc* d, DenseMix* out) {
+  const int K = d->K;
+  for (int m = 0; m < K; ++m)
+    for (int n = 0; n < K; ++n) out->Wt[n * K + m] = d->W[m * K + n];
+}
+
+// CTAs per SM for (kernel, block, smem); raises the dynamic shared-memory limit when needed.
+template <typename Kern>
+int ctas_per_sm(fgd_ctx* c, Kern kern, int block, size_t smem, int* out) {
+  const auto key = std::make_pair(reinterpret_cast<const void*>(kern), smem);
+  auto it = c->occupancy.find(key);
+  if (it != c->occupancy.end()) {
+    *out = it->second;
+    return FGD_OK;
+  }
+  if (smem > 48 * 1024)
+    FGD_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  int n = 0;
+  FGD_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, block, smem));
+  if (n < 1) return fail(c, FGD_ERR_UNSUPPORTED, "kernel does not fit on an SM (smem %zu B)", smem);
+  c->occupancy[key] = n;
+  *out = n;
+  return FGD_OK;
+}
+
+template <typename Kern>
+int persistent_grid(fgd_ctx* c, Kern kern, int block, size_t smem, int64_t ntiles, int* grid) {
+  int per_sm = 0;
+  if (int rc = ctas_per_sm(c, kern, block, smem, &per_sm)) return rc;
+  int64_t g = (int64_t)per_sm * c->num_sms;
+  if (g > ntiles) g = ntiles;
+  if (g > kMaxPartialBlocks) g = kMaxPartialBlocks;
+  if (g < 1) g = 1;
+  *grid = (int)g;
+  return FGD_OK;
+}
+
+int check_launch(fgd_ctx* c, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(c, e, what);
+  c->launches += 1;
+  return FGD_OK;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
+    else if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+// ---- compile-time K / vector width selection -------------------------------------------
+// KT = K for the instantiated worker counts, 0 (runtime-K generic kernel) otherwise.
+int kt_of(int K) {
+  switch (K) {
+    case 2: case 4: case 8: case 16: case 32: case 64: return K;
+    default: return 0;
+  }
+}
+int want_vec(int KT) { return KT == 0 ? 1 : (KT <= 16 ? 4 : (KT == 32 ? 2 : 1)); }
+
+// Calls f.template operator()<KT, VEC>() for the (KT, VEC) pair chosen at run time.
+template <typename F>
+int dispatch_kv(int KT, int VEC, F&& f) {
+#define FGD_CASE(kt, v) \
+  if (KT == kt && VEC == v) return f.template operator()<kt, v>();
+  FGD_CASE(0, 1)
+  FGD_CASE(2, 4) FGD_CASE(2, 2) FGD_CASE(2, 1)
+  FGD_CASE(4, 4) FGD_CASE(4, 2) FGD_CASE(4, 1)
+  FGD_CASE(8, 4) FGD_CASE(8, 2) FGD_CASE(8, 1)
+  FGD_CASE(16, 4) FGD_CASE(16, 2) FGD_CASE(16, 1)
+  FGD_CASE(32, 2) FGD_CASE(32, 1)
+  FGD_CASE(64, 1)
+#undef FGD_CASE
+  return FGD_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+#endif

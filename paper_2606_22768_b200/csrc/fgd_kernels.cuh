@@ -179,19 +179,21 @@ __device__ __forceinline__ float p_hsum(const Pack<VEC>& a) {
 
 // Gather of a mix row from a thread-private shared column:
 //   out = w_self[m] * col[m] + sum_{j < D} w[m][j] * col[nbr[m][j]]
-template <int VEC, int BLOCK>
+// DT >= 0: the number of neighbour slots is a compile-time constant (fully unrolled, every
+// index and weight a constant-bank operand, loads of all rows schedulable together);
+// DT < 0: D is read at run time (warp-uniform loop).
+template <int VEC, int BLOCK, int DT = -1>
 __device__ __forceinline__ Pack<VEC> gather_row(const GatherMix& mx, int m, const float* col, int tid) {
-  Pack<VEC> acc;
-  const Pack<VEC> self = SCol<VEC>::ld(col, m * BLOCK + tid);
-  acc = p_mul<VEC>(self, mx.w_self[m]);
-  // D is warp-uniform: a real loop issues D slots, where an unrolled predicated one would
-  // issue all FGD_MAX_D of them
-  const int D = mx.D;
+  Pack<VEC> acc = p_mul<VEC>(SCol<VEC>::ld(col, m * BLOCK + tid), mx.w_self[m]);
+  if constexpr (DT >= 0) {
+#pragma unroll
+    for (int j = 0; j < DT; ++j)
+      acc = p_fma<VEC>(SCol<VEC>::ld(col, mx.nbr[m * FGD_MAX_D + j] * BLOCK + tid), mx.w[m * FGD_MAX_D + j], acc);
+  } else {
+    const int D = mx.D;
 #pragma unroll 1
-  for (int j = 0; j < D; ++j) {
-    const int n = mx.nbr[m * FGD_MAX_D + j];
-    const float wj = mx.w[m * FGD_MAX_D + j];
-    acc = p_fma<VEC>(SCol<VEC>::ld(col, n * BLOCK + tid), wj, acc);
+    for (int j = 0; j < D; ++j)
+      acc = p_fma<VEC>(SCol<VEC>::ld(col, mx.nbr[m * FGD_MAX_D + j] * BLOCK + tid), mx.w[m * FGD_MAX_D + j], acc);
   }
   return acc;
 }

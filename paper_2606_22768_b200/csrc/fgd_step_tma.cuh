@@ -75,7 +75,9 @@ __host__ __device__ inline size_t tma_stage_bytes(int K, int T, int n_tensors) {
 
 constexpr int kMaxStages = 8;
 
-template <int KT, int VEC, int CONSUMERS, bool DENSE2, typename M2>
+// D2T: compile-time neighbour count of a gather Mix2 (-1 = read at run time; ignored for a mean
+// or dense Mix2).
+template <int KT, int VEC, int CONSUMERS, bool DENSE2, int D2T, typename M2>
 __global__ void __launch_bounds__(CONSUMERS + 32)
 outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
                       const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
@@ -274,7 +276,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           for (int m = 0; m < K; ++m) {
             Pack<VEC> gh;
             if (m2.kind == KMIX_MEAN) gh = gmean;
-            else gh = gather_row<VEC, TPB>(m2, m, B, t);
+            else gh = gather_row<VEC, TPB, D2T>(m2, m, B, t);
             finish_row(m, gh);
           }
         }

@@ -1,0 +1,18 @@
+// Interface between the entry points and the TMA-pipelined fused-step launcher.
+#ifndef FGD_STEP_TMA_H_
+#define FGD_STEP_TMA_H_
+
+#include <cuda_runtime.h>
+
+#include "fgd_internal.h"
+
+struct fgd_ctx;
+struct FgdTmaShape {
+  int vec, consumers, stages;
+};
+// Can the TMA kernel run this call?  Picks the tile shape.
+bool fgd_tma_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, FgdTmaShape* out);
+int fgd_launch_step_tma(fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g2,
+                        const fgd::DenseMix& d2, const fgd::GatherMix& g1, FgdTmaShape shape, cudaStream_t st,
+                        int* grid_out);
+#endif
