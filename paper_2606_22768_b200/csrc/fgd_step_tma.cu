@@ -30,6 +30,13 @@ int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc) {
   return FGD_OK;
 }
 
+// Tensors per stage: theta_prev, theta_local, momentum, plus a matrix-valued Mix1 result only in
+// the kernels that cannot keep it in registers (run-time K, dense Mix2 with K > 16).
+int tma_n_tensors(const StepArgs& a, int KT, bool dense2) {
+  const bool xregs = KT > 0 && !(dense2 && KT > 16);
+  return (a.xsrc == XSRC_MATRIX && !xregs) ? 4 : 3;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Tile shapes of the TMA kernel.  A stage holds n_tensors x K x (consumers * vec) floats and at
@@ -59,7 +66,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* ou
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
-  const int K = c->K, KT = kt_of(K), NT = a.xsrc == XSRC_MATRIX ? 4 : 3;
+  const int K = c->K, KT = kt_of(K), NT = tma_n_tensors(a, KT, dense2);
   const size_t budget = (size_t)c->max_smem_optin - 4096;  // static shared memory + slack
   for (const auto& sh : kTmaShapes) {
     if (sh[0] != KT) continue;
@@ -82,7 +89,7 @@ int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix&
   TmaStepArgs ta;
   ta.s = a;
   ta.status = c->status;
-  ta.n_tensors = a.xsrc == XSRC_MATRIX ? 4 : 3;
+  ta.n_tensors = tma_n_tensors(a, KT, dense2);
   ta.stages = sh.stages;
   const int T = sh.consumers * sh.vec;
   const int boxc = T < 256 ? T : 256;

@@ -170,8 +170,31 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
     }
     const float invK = 1.0f / (float)K;
     const float lr = a.lr, mu = a.mu;
+    // A matrix-valued Mix1 result is used only by the thread that owns the column, so with a
+    // compile-time K it is not staged: each thread prefetches its K rows of the NEXT tile
+    // straight into registers while it works on the current one (a whole tile of lead time).
+    constexpr bool XREGS = (KT > 0) && !(DENSE2 && KT > 16);
+    constexpr int KX = XREGS ? KT : 1;
+    const bool x_direct = XREGS && a.xsrc == XSRC_MATRIX;
+    Pack<VEC> xr[KX], xr_next[KX];
+    auto fetch_x = [&](int64_t tile_, Pack<VEC> (&dst)[KX]) {
+      const int64_t c_ = tile_ * T + (int64_t)tid * VEC;
+      if (tile_ < ntiles && c_ + VEC <= P) {
+#pragma unroll
+        for (int m = 0; m < KX; ++m) dst[m] = ld_stream<VEC>(a.x + (size_t)m * ld + c_);
+      } else if (tile_ < ntiles && c_ < P) {
+        for (int m = 0; m < KX; ++m)
+          for (int q = 0; q < VEC; ++q) dst[m].v[q] = c_ + q < P ? a.x[(size_t)m * ld + c_ + q] : 0.f;
+      }
+    };
+    if (x_direct) fetch_x(blockIdx.x, xr_next);
     int64_t i = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
+      if (x_direct) {
+#pragma unroll
+        for (int m = 0; m < KX; ++m) xr[m] = xr_next[m];
+        fetch_x(tile + gridDim.x, xr_next);
+      }
       const int s = (int)(i % STAGES);
       const uint32_t use = (uint32_t)(i / STAGES);
       const int64_t col = tile * T + (int64_t)tid * VEC;
@@ -247,9 +270,14 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
         auto finish_row = [&](int m, const Pack<VEC>& gh) {
           const size_t off = (size_t)m * ld;
           Pack<VEC> xm;
-          if (a.xsrc == XSRC_MATRIX) xm = SCol<VEC>::ld(X, m * TPB + t);
-          else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) xm = gather_row<VEC, TPB>(m1, m, A, t);
-          else xm = xv;
+          if (a.xsrc == XSRC_MATRIX) {
+            if constexpr (XREGS) xm = xr[m];
+            else xm = SCol<VEC>::ld(X, m * TPB + t);
+          } else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) {
+            xm = gather_row<VEC, TPB>(m1, m, A, t);
+          } else {
+            xm = xv;
+          }
           Pack<VEC> v;
           if constexpr (REGS) v = av[m];
           else v = SCol<VEC>::ld(C, m * TPB + t);
