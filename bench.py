@@ -291,7 +291,8 @@ def run_ours(args):
     achieved = step_bytes / (kern_ms * 1e-3) / 1e9
     tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if tr is None else tr * K * P, "kernel": "outer_step_tma_kernel",
+                "traffic": None if tr is None else tr * K * P,
+                "kernel": "outer_step_dense_tc_kernel" if (cfg["mix2"][0] == "dense" and K == 64) else "outer_step_tma_kernel",
                 "kernel_ms": kern_ms, "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
                 "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / 8000.0}

@@ -71,11 +71,13 @@ int fgd_destroy(fgd_ctx* ctx);
  * last failing fgd_create / host helper on this thread.  The string is owned by the library. */
 const char* fgd_last_error(const fgd_ctx* ctx);
 const char* fgd_status_string(int status);
-/* Which kernel family fgd_outer_step uses.  AUTO (default): the TMA-pipelined kernel when the
+/* Which kernel family fgd_outer_step uses.  AUTO (default): a TMA-pipelined kernel when the
  * tensors allow it (16-byte aligned bases, ld % 4 == 0, two pipeline stages fit in shared
- * memory), else the register kernel.  REGISTER / TMA force one (TMA fails with
- * FGD_ERR_UNSUPPORTED when not eligible).  Both compute the same round. */
-typedef enum { FGD_PATH_AUTO = 0, FGD_PATH_REGISTER = 1, FGD_PATH_TMA = 2 } fgd_path;
+ * memory), else the register kernel; a dense Mix2 with K = 64 runs its contraction on the
+ * tensor cores (3 x TF32, fp32 accumulate) when Mix1 is the mean.  REGISTER / TMA force a
+ * family (TMA fails with FGD_ERR_UNSUPPORTED when not eligible); TMA_FP32 is TMA with the
+ * dense contraction kept on the fp32 CUDA cores.  All compute the same round. */
+typedef enum { FGD_PATH_AUTO = 0, FGD_PATH_REGISTER = 1, FGD_PATH_TMA = 2, FGD_PATH_TMA_FP32 = 3 } fgd_path;
 int fgd_set_path(fgd_ctx* ctx, int path);
 /* Synchronises `stream` and reports whether any kernel of this context abandoned a bounded
  * device-side wait since the last check: FGD_OK, or FGD_ERR_TIMEOUT (then the outputs of the

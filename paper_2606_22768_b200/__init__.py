@@ -34,7 +34,7 @@ FGD_ERR_TIMEOUT = -6
 
 FGD_MIX_IDENTITY, FGD_MIX_MEAN, FGD_MIX_SPARSE, FGD_MIX_DENSE = 0, 1, 2, 3
 FGD_RENORM_NONE, FGD_RENORM_SELF_ABSORB, FGD_RENORM_METROPOLIS = 0, 1, 2
-FGD_PATH_AUTO, FGD_PATH_REGISTER, FGD_PATH_TMA = 0, 1, 2
+FGD_PATH_AUTO, FGD_PATH_REGISTER, FGD_PATH_TMA, FGD_PATH_TMA_FP32 = 0, 1, 2, 3
 
 
 class FgdError(RuntimeError):

@@ -16,7 +16,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfgd.so")
 SOURCES = ["fgd_api.cu", "fgd_step_tma.cu", "fgd_noalloc.cu", "fgd_host.cpp"]
-HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_step_tma.h", "fgd_ctx.h", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
+HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_step_dense_tc.cuh", "fgd_step_tma.h", "fgd_ctx.h", "fgd_internal.h", os.path.join(ROOT, "include", "fgd.h")]
 
 NVCC_FLAGS = ["-std=c++20", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include")]

@@ -74,7 +74,7 @@ const char* fgd_last_error(const fgd_ctx* c) { return c ? c->err : g_thread_erro
 
 int fgd_set_path(fgd_ctx* c, int path) {
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_set_path: ctx is NULL");
-  if (path < FGD_PATH_AUTO || path > FGD_PATH_TMA) return fail(c, FGD_ERR_INVALID_ARG, "fgd_set_path: unknown path %d", path);
+  if (path < FGD_PATH_AUTO || path > FGD_PATH_TMA_FP32) return fail(c, FGD_ERR_INVALID_ARG, "fgd_set_path: unknown path %d", path);
   c->path = path;
   return FGD_OK;
 }
@@ -223,10 +223,13 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
   int rc = FGD_OK;
   FgdTmaShape shape{0, 0, 0};
   const bool can_tma = fgd_tma_eligible(c, a, dense2, &shape);
-  if (c->path == FGD_PATH_TMA && !can_tma)
+  const bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, dense2, g1);
+  if ((c->path == FGD_PATH_TMA || c->path == FGD_PATH_TMA_FP32) && !can_tma)
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
-  if (can_tma && c->path != FGD_PATH_REGISTER) {
+  if (can_tc && c->path != FGD_PATH_REGISTER) {
+    rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
+  } else if (can_tma && c->path != FGD_PATH_REGISTER) {
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x});

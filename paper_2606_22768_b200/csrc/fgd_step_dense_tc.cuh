@@ -1,0 +1,316 @@
+// Fused outer step with a DENSE Mix2 on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// For a dense K x K mixing matrix the step ghat[m][p] = sum_n W[m][n] g[n][p] really is a
+// contraction (2K flop per worker-parameter; at K = 64 the CUDA-core version is FMA-bound at
+// about a quarter of the HBM roofline).  Here it runs as tcgen05.mma.kind::tf32 with the
+// error-compensated three-product split
+//     W g  ~=  W_hi g_hi + W_hi g_lo + W_lo g_hi          (hi = tf32-rounded, lo = remainder)
+// accumulated in fp32 in tensor memory, which keeps the result within fp32 rounding of the
+// exact product (a single tf32 product would miss the 1e-5 parity bar).
+//
+// Mapping.  The 128 columns of a tile are the M dimension of the MMA, the K workers n are its
+// K dimension and the K output rows m its N dimension:
+//     D[col][m] += A[col][n] * B[n][m],   A = g^T, B = W^T, both K-major (worker-contiguous).
+// D row `col` lives in TMEM lane `col`, so after tcgen05.ld thread `col` holds ghat[0..K-1] of
+// ITS column in registers -- the same thread-owns-a-column layout as the other kernels; the
+// Nesterov update, the streaming stores and the consensus sums follow without any exchange.
+//
+// Pipeline per CTA (one per SM): a producer warp streams [K x 128] boxes of theta_prev,
+// theta_local and momentum into a 2-stage shared-memory ring with 2-D TMA loads; the four
+// consumer warps compute g = theta_prev - theta_local in registers, split it and write g_hi /
+// g_lo IN PLACE over the theta_local / theta_prev boxes of the stage in the K-major core-matrix
+// operand layout (a thread's four consecutive workers are one 16-byte row of a core matrix, so
+// its stores are 128-bit and conflict-free); one thread issues the 3 x (K/8) MMAs and commits them to an
+// mbarrier; every consumer then reads its accumulator row from TMEM.
+// All waits are bounded; tensor memory is always released before the kernel returns.
+#ifndef FGD_STEP_DENSE_TC_CUH_
+#define FGD_STEP_DENSE_TC_CUH_
+
+#include "fgd_step_tma.cuh"
+
+namespace fgd {
+
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ float to_tf32(float x) {   // round to nearest tf32 (low 13 mantissa bits zero)
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
+// Shared-memory matrix descriptor of the tcgen05 MMA (addresses and offsets in 16-byte units).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
+  d |= (uint64_t)(layout_type & 7) << 61;  // 0 = no swizzle, 2 = 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 bit x 64 columns: thread i of the warp receives columns 0..63 of lane (base + i).
+__device__ __forceinline__ void tmem_ld_64(uint32_t taddr, float (&r)[64]) {
+  uint32_t* u = reinterpret_cast<uint32_t*>(r);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+        "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+        "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31]),
+        "=r"(u[32]), "=r"(u[33]), "=r"(u[34]), "=r"(u[35]), "=r"(u[36]), "=r"(u[37]), "=r"(u[38]), "=r"(u[39]),
+        "=r"(u[40]), "=r"(u[41]), "=r"(u[42]), "=r"(u[43]), "=r"(u[44]), "=r"(u[45]), "=r"(u[46]), "=r"(u[47]),
+        "=r"(u[48]), "=r"(u[49]), "=r"(u[50]), "=r"(u[51]), "=r"(u[52]), "=r"(u[53]), "=r"(u[54]), "=r"(u[55]),
+        "=r"(u[56]), "=r"(u[57]), "=r"(u[58]), "=r"(u[59]), "=r"(u[60]), "=r"(u[61]), "=r"(u[62]), "=r"(u[63])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+constexpr int kTcK = 64;            // workers (MMA K and N dimensions)
+constexpr int kTcCols = 128;        // columns per tile (MMA M dimension) = consumer threads
+constexpr int kTcStages = 2;
+constexpr int kTcTmemCols = 64;     // fp32 accumulator columns (= K), a power of two >= 32
+constexpr uint32_t kTcBox = kTcK * kTcCols * sizeof(float);   // 32 KB: one tensor of a stage
+constexpr uint32_t kTcWBytes = kTcK * kTcK * sizeof(float);   // 16 KB: one split of W
+// dynamic shared memory: 1 KB alignment slack + stages + W_hi + W_lo
+constexpr size_t kTcSmem = 1024 + (size_t)kTcStages * 3 * kTcBox + 2 * kTcWBytes;
+
+__global__ void __launch_bounds__(kTcCols + 32)
+outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
+                           const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
+                           const __grid_constant__ CUtensorMap tm_mom) {
+  constexpr int K = kTcK, T = kTcCols, STAGES = kTcStages;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];   // full[], empty[], mma
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_slot;
+
+  const StepArgs& a = ta.s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool want_cd = a.partials != nullptr;
+  // operand regions on 1024-byte boundaries
+  unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* wb_hi = base + (size_t)STAGES * 3 * kTcBox;
+  unsigned char* wb_lo = wb_hi + kTcWBytes;
+  const uint32_t mma_bar = smem_u32(&bars[2 * STAGES]);
+
+  const int64_t P = a.P, ld = a.ld;
+  const int64_t ntiles = (P + T - 1) / T;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&bars[s]), 1);
+      mbar_init(smem_u32(&bars[STAGES + s]), T);
+    }
+    mbar_init(mma_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // B operand = W^T as an N x K (m x n) matrix, K-major, no swizzle: 8-row x 16-byte core
+  // matrices; core matrices adjacent in K are 128 B apart, adjacent in N 2048 B apart.
+  for (int i = tid; i < K * K; i += T + 32) {
+    const int n = i / K, m = i % K;          // m2.Wt[n*K+m] = W[m][n]
+    const float w = m2.Wt[i];
+    const float hi = to_tf32(w);
+    const uint32_t off = (uint32_t)(m >> 3) * 2048u + (uint32_t)(n >> 2) * 128u + (uint32_t)(m & 7) * 16u + (uint32_t)(n & 3) * 4u;
+    *reinterpret_cast<float*>(wb_hi + off) = hi;
+    *reinterpret_cast<float*>(wb_lo + off) = w - hi;
+  }
+  if (warp == T / 32) {   // the producer warp owns tensor memory: allocate K accumulator columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTcTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // W operands are read by the MMA (async proxy)
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+
+  float sacc[K];
+#pragma unroll
+  for (int m = 0; m < K; ++m) sacc[m] = 0.f;
+
+  if (warp == T / 32) {
+    // ===================================================== producer (one elected lane)
+    if (lane == 0) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      int64_t i = 0;
+      bool ok = true;
+      for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
+        const int s = (int)(i % STAGES);
+        const uint32_t use = (uint32_t)(i / STAGES);
+        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1);
+        if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
+        const uint32_t full = smem_u32(&bars[s]);
+        mbar_expect_tx(full, 3 * kTcBox);
+        const uint32_t dst = smem_u32(base + (size_t)s * 3 * kTcBox);
+        const int c0 = (int)(tile * T);
+        tma_load_2d(dst, &tm_prev, c0, 0, full, policy);
+        tma_load_2d(dst + kTcBox, &tm_local, c0, 0, full, policy);
+        tma_load_2d(dst + 2 * kTcBox, &tm_mom, c0, 0, full, policy);
+      }
+      if (!ok) {
+        *(volatile int*)&abort_flag = 1;
+        atomicExch(ta.status, FGD_ERR_TIMEOUT);
+        for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
+          mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1);
+      }
+    }
+  } else {
+    // ===================================================== consumers: thread t owns column t of the tile
+    const float invK = 1.0f / (float)K;
+    const float lr = a.lr, mu = a.mu;
+    const bool need_tsum = a.xsrc == XSRC_FUSED;                      // fused mean Mix1
+    // A operand = g^T as an M x K (column x worker) matrix, K-major, no swizzle, same core-matrix
+    // scheme as B: row `tid`, four consecutive workers = one 16-byte core-matrix row, so a
+    // thread's 64 values go out as 16 conflict-free 128-bit stores.
+    const uint32_t op_row = (uint32_t)(tid >> 3) * 2048u + (uint32_t)(tid & 7) * 16u;
+    // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
+    constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
+    int64_t i = 0;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
+      const int s = (int)(i % STAGES);
+      const uint32_t use = (uint32_t)(i / STAGES);
+      const int64_t col = tile * T + tid;
+      const bool live = col < P;
+      float xv = 0.f;
+      if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
+      unsigned char* stage = base + (size_t)s * 3 * kTcBox;
+      float* A = reinterpret_cast<float*>(stage);                 // theta_prev  -> g_lo operand
+      float* B = reinterpret_cast<float*>(stage + kTcBox);        // theta_local -> g_hi operand
+      float* C = reinterpret_cast<float*>(stage + 2 * kTcBox);    // momentum
+      // ---- phase 1: g for all workers in registers
+      float g[K];
+      float tsum = 0.f;
+      const bool got = mbar_wait(smem_u32(&bars[s]), use & 1);
+      if (got) {
+#pragma unroll
+        for (int n = 0; n < K; ++n) {
+          const float tp = A[n * T + tid];
+          g[n] = tp - B[n * T + tid];
+          if (need_tsum) tsum += tp;
+        }
+      } else {
+        *(volatile int*)&abort_flag = 1;
+        atomicExch(ta.status, FGD_ERR_TIMEOUT);
+      }
+      named_bar_sync(1, T);                       // every consumer has read its theta_prev / theta_local
+      if (*(volatile int*)&abort_flag) break;     // uniform: the flag was written before the barrier
+      // ---- operands: g_hi over the theta_local box, g_lo over the theta_prev box
+#pragma unroll
+      for (int n = 0; n < K; n += 4) {
+        float4 hi, lo;
+        hi.x = to_tf32(g[n]);     lo.x = g[n] - hi.x;
+        hi.y = to_tf32(g[n + 1]); lo.y = g[n + 1] - hi.y;
+        hi.z = to_tf32(g[n + 2]); lo.z = g[n + 2] - hi.z;
+        hi.w = to_tf32(g[n + 3]); lo.w = g[n + 3] - hi.w;
+        const uint32_t off = op_row + (uint32_t)(n >> 2) * 128u;
+        *reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(B) + off) = hi;
+        *reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(A) + off) = lo;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      named_bar_sync(2, T);                       // operands complete; last tile's TMEM reads are done too
+      if (tid == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_hi = smem_u32(B), a_lo = smem_u32(A);
+        const uint32_t b_hi = smem_u32(wb_hi), b_lo = smem_u32(wb_lo);
+#pragma unroll
+        for (int prod = 0; prod < 3; ++prod) {     // W_hi g_hi, W_hi g_lo, W_lo g_hi
+          const uint32_t aa = prod == 1 ? a_lo : a_hi;
+          const uint32_t bb = prod == 2 ? b_lo : b_hi;
+#pragma unroll
+          for (int ks = 0; ks < K / 8; ++ks) {
+            const uint64_t da = umma_desc(aa + (uint32_t)ks * 256u, 128u, 2048u, 0u);
+            const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, 2048u, 0u);
+            umma_tf32(tmem_base, da, db, idesc, (prod | ks) ? 1u : 0u);
+          }
+        }
+        umma_commit(mma_bar);
+      }
+      // ---- while the tensor core works: this column's momentum from the stage
+      float v[K];
+#pragma unroll
+      for (int m = 0; m < K; ++m) v[m] = C[m * T + tid];
+      if (a.xsrc != XSRC_VECTOR) xv = tsum * invK;
+      if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
+        *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
+        atomicExch(ta.status, FGD_ERR_TIMEOUT);
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float gh[K];
+      tmem_ld_64(tmem_base + ((uint32_t)(warp * 32) << 16), gh);
+      // ---- phase 2: Nesterov step for every worker of this column, stream out
+      float asum = 0.f;
+      if (live) {
+        float* const mom_col = a.momentum + col;
+        float* const new_col = a.theta_new + col;
+#pragma unroll
+        for (int m = 0; m < K; ++m) {
+          const float vn = fmaf(mu, v[m], gh[m]);
+          const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xv);
+          __stcs(mom_col + (size_t)m * ld, vn);
+          __stcs(new_col + (size_t)m * ld, tn);
+          v[m] = tn;
+          asum += tn;
+        }
+        if (want_cd) {
+          const float mean = asum * invK;
+#pragma unroll
+          for (int m = 0; m < K; ++m) {
+            const float d = v[m] - mean;
+            sacc[m] = fmaf(d, d, sacc[m]);
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&bars[STAGES + s]));
+    }
+  }
+
+  // ---- wrap-up: tensor memory back, consensus partial sums (stage memory is free now)
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == T / 32) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTcTmemCols) : "memory");
+  }
+  if (want_cd) {
+    double* red = reinterpret_cast<double*>(base);    // [T/32][K]
+    if (warp < T / 32) {
+#pragma unroll
+      for (int m = 0; m < K; ++m) {
+        double d = (double)sacc[m];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
+        if (lane == 0) red[warp * K + m] = d;
+      }
+    }
+    __syncthreads();
+    if (tid < K) {
+      double d = 0.0;
+#pragma unroll
+      for (int w = 0; w < T / 32; ++w) d += red[w * K + tid];
+      a.partials[(size_t)blockIdx.x * K + tid] = d;
+    }
+  }
+}
+
+}  // namespace fgd
+#endif

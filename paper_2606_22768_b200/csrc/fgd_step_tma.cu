@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include "fgd_ctx.h"
+#include "fgd_step_dense_tc.cuh"
 #include "fgd_step_tma.cuh"
 #include "fgd_step_tma.h"
 
@@ -141,6 +142,35 @@ int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix&
 }
 
 }  // namespace
+
+// Tensor-core dense step: K = 64, Mix1 given as the averaged row or fused as a mean.
+bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g1) {
+  if (!dense2 || c->K != kTcK || !c->encode_tiled) return false;
+  if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
+  if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
+  if (!(a.xsrc == XSRC_VECTOR || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
+  return (size_t)c->max_smem_optin >= kTcSmem + 1024;
+}
+
+int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, const GatherMix& g1, cudaStream_t st,
+                             int* grid_out) {
+  TmaStepArgs ta;
+  ta.s = a;
+  ta.status = c->status;
+  ta.n_tensors = 3;
+  ta.stages = kTcStages;
+  CUtensorMap tp, tl, tm;
+  if (int rc = make_tensor_map(c, &tp, a.theta_prev, kTcCols)) return rc;
+  if (int rc = make_tensor_map(c, &tl, a.theta_local, kTcCols)) return rc;
+  if (int rc = make_tensor_map(c, &tm, a.momentum, kTcCols)) return rc;
+  const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
+  int grid = 0;
+  auto kern = outer_step_dense_tc_kernel;
+  if (int r = persistent_grid(c, kern, kTcCols + 32, kTcSmem, ntiles, &grid)) return r;
+  kern<<<grid, kTcCols + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  *grid_out = grid;
+  return check_launch(c, "outer_step_dense_tc_kernel");
+}
 
 bool fgd_tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, FgdTmaShape* out) {
   TmaShape sh{0, 0, 0};
