@@ -126,6 +126,32 @@ def outer_round(W1, W2, theta_prev, theta_local, v, gamma: float = 0.7, mu: floa
     return (out, v, x, gh) if want_intermediates else (out, v)
 
 
+def outer_round_ex(W1, W2, theta_prev, theta_local, v, gamma: float = 0.7, mu: float = 0.9,
+                   mix2_ranges=None, average_momentum: bool = False):
+    """One outer round of the two variants the paper adds on top of Algorithm 1, composed from
+    the same one-equation primitives in the paper's order.
+
+    mix2_ranges: list of (lo, hi) column ranges.  Mix2 is applied only to columns inside a range
+        (the "-subset" configurations: Mix2 on a chosen subset of parameter blocks, "the rest pass
+        through identity", App. A); None = every column.
+    average_momentum: the GlobalM1S variants (App. B): Mix1 "also includes outer optimizer
+        state", i.e. v_m <- Mix1(v)_m before the Nesterov update.
+    Returns (theta_new, v_new).
+    """
+    tp, tl = _f64(theta_prev), _f64(theta_local)
+    K, P = tp.shape
+    x = mix(W1, tp)
+    g = outer_grad(tp, tl)
+    ghat = mix(W2, g)
+    if mix2_ranges is not None:
+        inside = np.zeros(P, dtype=bool)
+        for lo, hi in mix2_ranges:
+            inside[int(lo):int(hi)] = True
+        ghat[:, ~inside] = g[:, ~inside]
+    v_in = mix(W1, v) if average_momentum else _f64(v)
+    return nesterov(x, ghat, v_in, gamma, mu)
+
+
 def consensus_sumsq(theta) -> np.ndarray:
     """s[m] = sum_p (theta[m][p] - mean_p)^2."""
     th = _f64(theta)

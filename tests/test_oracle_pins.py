@@ -405,3 +405,43 @@ def test_expected_consensus_distance_closed_form():
     expect = P * GAMMA ** 2 * (1 + MU) ** 2 * sigma ** 2 * (1.0 / 3.0) / K
     assert expect == pytest.approx(0.154569, rel=1e-5)
     assert cd_sq == pytest.approx(expect, rel=6e-3)
+
+
+# ------------------------------------------------------------------ variants: subset Mix2, momentum averaging
+def test_subset_mix2_limits_and_brute_force():
+    K, P = 4, 12
+    W1, W2 = oracle.dense_W("mean", K), _ring_W(K)
+    tp, tl, v = _rand(K, P, 1, 0.02), _rand(K, P, 2, 0.02), _rand(K, P, 3, 1e-3)
+    full = oracle.outer_round(W1, W2, tp, tl, v, GAMMA, MU)
+    ident = oracle.outer_round(W1, oracle.dense_W("identity", K), tp, tl, v, GAMMA, MU)
+    every = oracle.outer_round_ex(W1, W2, tp, tl, v, GAMMA, MU, mix2_ranges=[(0, P)])
+    none = oracle.outer_round_ex(W1, W2, tp, tl, v, GAMMA, MU, mix2_ranges=[(0, 0)])
+    assert np.array_equal(every[0], full[0]) and np.array_equal(every[1], full[1])
+    assert np.array_equal(none[0], ident[0]) and np.array_equal(none[1], ident[1])
+    # columns 4..7 and 10..11 mixed, the rest identity: column by column it is one or the other
+    sub = oracle.outer_round_ex(W1, W2, tp, tl, v, GAMMA, MU, mix2_ranges=[(4, 8), (10, 12)])
+    for p in range(P):
+        src = full if (4 <= p < 8 or p >= 10) else ident
+        assert np.array_equal(sub[0][:, p], src[0][:, p]) and np.array_equal(sub[1][:, p], src[1][:, p])
+
+
+def test_momentum_averaging_reproduces_diloco_trajectory():
+    """Mix1 = global average of parameters AND momentum, no Mix2: the averaged model follows
+    DiLoCo's trajectory exactly (Sec. 4.2 with the state synchronised as App. B requires):
+    x_{r+1} = mean_m z_{m,r+1} = OuterOpt(x_r, -mean_m Delta_{m,r})."""
+    K, P, R = 8, 30, 4
+    J, I = oracle.dense_W("mean", K), oracle.dense_W("identity", K)
+    base = _rand(1, P, 1, 0.02)
+    z = np.repeat(base, K, axis=0)
+    v = np.zeros((K, P))
+    drifts = [_rand(K, P, 20 + r, 1e-3) for r in range(R)]
+    means = []
+    for r in range(R):
+        z, v = oracle.outer_round_ex(J, I, z, z + drifts[r], v, GAMMA, MU, average_momentum=True)
+        means.append(z.mean(0))
+    ref = _torch_nesterov_steps(base[0], [-drifts[r].mean(0) for r in range(R)])
+    for r in range(R):
+        np.testing.assert_allclose(means[r], ref[r], rtol=1e-12, atol=1e-16)
+    # without the momentum averaging the per-worker states differ, with it Mix1(v) is common
+    z2, v2 = oracle.outer_round_ex(J, I, z, z + drifts[0], v, GAMMA, MU, average_momentum=False)
+    assert np.abs(v2 - v2.mean(0)).max() > 1e-6
