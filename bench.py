@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--config", type=int, default=3, choices=sorted(CONFIGS))
     ap.add_argument("--cols", type=int, default=0,
                     help="profiling only: shrink P to this many columns (same kernels, smaller launch)")
+    ap.add_argument("--subset-frac", type=float, default=0.0,
+                    help="variant: restrict Mix2 to about this fraction of the columns (three blocks)")
+    ap.add_argument("--average-momentum", action="store_true", help="variant: GlobalM1S (needs Mix1 = mean)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -245,6 +248,15 @@ def run_ours(args):
     cd_log = torch.zeros((warmup + steps + 8, K), dtype=torch.float64, device=dev)
     main = torch.cuda.current_stream(dev)
 
+    ranges = None
+    if args.subset_frac > 0.0:      # three blocks (embeddings, LM head, first layers), 4-column bounds
+        f = args.subset_frac
+        q = lambda t: int(t * P) // 4 * 4
+        ranges = [(0, q(0.4 * f)), (q(0.5), q(0.5 + 0.3 * f)), (q(1.0 - 0.3 * f), P)]
+        cfg["name"] += f" [variant: Mix2 on {sum(b - a for a, b in ranges) / P:.0%} of the columns]"
+    if args.average_momentum:
+        cfg["name"] += " [variant: momentum averaged (GlobalM1S)]"
+
     def one_round(r, ev_pair=None):
         m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
         m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
@@ -253,7 +265,7 @@ def run_ours(args):
         if ev_pair is not None:
             main.wait_event(drv._pending[0])     # keep the Mix1 wait out of the kernel's event pair
             ev_pair[0].record(main)
-        drv.step(m2, local, theta, mom, theta, 0.7, 0.9)
+        drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix2_ranges=ranges, average_momentum=args.average_momentum)
         if ev_pair is not None:
             ev_pair[1].record(main)
 

@@ -50,6 +50,7 @@ extern "C" {
 
 #define FGD_MAX_K 64 /* most workers (rows) */
 #define FGD_MAX_D 8  /* most neighbour slots per worker in a sparse mix */
+#define FGD_MAX_RANGES 8 /* most column ranges of a subset Mix2 */
 
 typedef enum {
   FGD_OK = 0,
@@ -149,6 +150,26 @@ int fgd_outer_step(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* m
                    const float* x, int x_is_vector, const float* theta_local,
                    const float* theta_prev, float* momentum, float* theta_new, double lr,
                    double mu, double* cd_sumsq, void* stream);
+
+/* The two variants the paper adds to Algorithm 1, as options of the same fused step.
+ *   mix2_ranges / n_ranges  the "-subset" configurations (Sec. 4.1, App. A): Mix2 is applied only
+ *       to columns p with lo <= p < hi for one of the n_ranges (<= FGD_MAX_RANGES) host pairs
+ *       {lo, hi} in mix2_ranges[2*n_ranges]; every other column passes through identity.
+ *       Bounds must be multiples of 4 columns (hi may also be P).  n_ranges = 0: every column.
+ *   average_momentum        the GlobalM1S configurations (App. B): Mix1 also averages the outer
+ *       optimizer state, v_m <- (1/K) sum_n v_n, before the Nesterov update.  Needs Mix1 to be
+ *       the global average (x given as the averaged row, or mix1_fused of kind MEAN), else
+ *       FGD_ERR_UNSUPPORTED.
+ * opts == NULL is fgd_outer_step. */
+typedef struct {
+  const int64_t* mix2_ranges;
+  int32_t n_ranges;
+  int32_t average_momentum;
+} fgd_step_options;
+int fgd_outer_step_ex(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused,
+                      const float* x, int x_is_vector, const float* theta_local,
+                      const float* theta_prev, float* momentum, float* theta_new, double lr,
+                      double mu, double* cd_sumsq, const fgd_step_options* opts, void* stream);
 
 /* s_m = sum_p (theta[m][p] - (1/K) sum_n theta[n][p])^2 into device cd_sumsq[K] (doubles).
  * The paper gives two L2 consensus distances, both functions of s: the mean of the

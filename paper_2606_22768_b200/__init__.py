@@ -68,6 +68,7 @@ def _load():
         "fgd_outer_grad": (i32, [vp, vp, vp, vp, vp]),
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
+        "fgd_outer_step_ex": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp, vp]),
         "fgd_consensus_distance": (i32, [vp, vp, vp, vp]),
         "fgd_consensus_distance_noalloc": (i32, [i32, i32, i64, i64, vp, vp, vp]),
         "fgd_topo_ring": (i32, [i32, vp, vp, vp]),
@@ -300,6 +301,30 @@ def fgd_outer_step(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x
         _dev_ptr(momentum, "momentum", "torch.float32"),
         _dev_ptr(theta_new, "theta_new", "torch.float32"), float(lr), float(mu),
         _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), _stream(stream)))
+
+
+class _CStepOptions(ctypes.Structure):
+    _fields_ = [("mix2_ranges", ctypes.c_void_p), ("n_ranges", ctypes.c_int32), ("average_momentum", ctypes.c_int32)]
+
+
+def fgd_outer_step_ex(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x, x_is_vector: bool,
+                      theta_local, theta_prev, momentum, theta_new, lr: float = 0.7, mu: float = 0.9,
+                      cd_sumsq=None, mix2_ranges=None, average_momentum: bool = False, stream=None) -> None:
+    """fgd_outer_step with the paper's two variants: Mix2 only inside the given (lo, hi) column
+    ranges (the "-subset" configurations) and/or the momentum averaged first (GlobalM1S)."""
+    ranges = None
+    if mix2_ranges is not None:
+        ranges = np.ascontiguousarray(np.asarray(mix2_ranges, dtype=np.int64).reshape(-1, 2))
+    opts = _CStepOptions(None if ranges is None else ranges.ctypes.data, 0 if ranges is None else ranges.shape[0],
+                         int(bool(average_momentum)))
+    ctx._check(_lib.fgd_outer_step_ex(
+        ctx._h, ctypes.byref(mix2.c()), None if mix1_fused is None else ctypes.byref(mix1_fused.c()),
+        _dev_ptr(x, "x", "torch.float32"), int(bool(x_is_vector)),
+        _dev_ptr(theta_local, "theta_local", "torch.float32"),
+        _dev_ptr(theta_prev, "theta_prev", "torch.float32"),
+        _dev_ptr(momentum, "momentum", "torch.float32"),
+        _dev_ptr(theta_new, "theta_new", "torch.float32"), float(lr), float(mu),
+        _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), ctypes.byref(opts), _stream(stream)))
 
 
 def fgd_consensus_distance(ctx: Context, theta, cd_sumsq, stream=None) -> None:

@@ -159,6 +159,14 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
 int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused, const float* x,
                    int x_is_vector, const float* theta_local, const float* theta_prev, float* momentum,
                    float* theta_new, double lr, double mu, double* cd_sumsq, void* stream) {
+  return fgd_outer_step_ex(c, mix2, mix1_fused, x, x_is_vector, theta_local, theta_prev, momentum, theta_new, lr, mu,
+                           cd_sumsq, nullptr, stream);
+}
+
+int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused, const float* x,
+                      int x_is_vector, const float* theta_local, const float* theta_prev, float* momentum,
+                      float* theta_new, double lr, double mu, double* cd_sumsq, const fgd_step_options* opts,
+                      void* stream) {
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_outer_step: ctx is NULL");
   if (!theta_local || !theta_prev || !momentum || !theta_new)
     return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_step: NULL tensor");
@@ -206,6 +214,26 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
   a.xsrc = mix1_fused ? XSRC_FUSED : (x_is_vector ? XSRC_VECTOR : XSRC_MATRIX);
   a.lr = (float)lr;
   a.mu = (float)mu;
+  a.n_ranges = 0;
+  a.avg_momentum = 0;
+  for (int i = 0; i < FGD_MAX_RANGES; ++i) a.range_lo[i] = a.range_hi[i] = 0;
+  if (opts) {
+    if (opts->n_ranges < 0 || opts->n_ranges > FGD_MAX_RANGES || (opts->n_ranges > 0 && !opts->mix2_ranges))
+      return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_step_ex: n_ranges=%d out of [0, %d] or ranges missing", opts->n_ranges, FGD_MAX_RANGES);
+    for (int i = 0; i < opts->n_ranges; ++i) {
+      const int64_t lo = opts->mix2_ranges[2 * i], hi = opts->mix2_ranges[2 * i + 1];
+      if (lo < 0 || hi < lo || hi > c->P || lo % 4 != 0 || (hi % 4 != 0 && hi != c->P))
+        return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_step_ex: range %d = [%lld, %lld) must lie in [0, P] on multiples of 4 columns", i, (long long)lo, (long long)hi);
+      a.range_lo[i] = lo;
+      a.range_hi[i] = hi;
+    }
+    a.n_ranges = opts->n_ranges;
+    if (opts->average_momentum) {
+      const bool mean1 = mix1_fused ? mix1_fused->kind == FGD_MIX_MEAN : (x_is_vector != 0);
+      if (!mean1) return fail(c, FGD_ERR_UNSUPPORTED, "fgd_outer_step_ex: average_momentum needs Mix1 to be the global average");
+      a.avg_momentum = 1;
+    }
+  }
 
   GatherMix g1, g2;
   memset(&g1, 0, sizeof(g1));

@@ -48,7 +48,24 @@ struct StepArgs {
   int stage_tp;         // 1 when Mix1 is a fused gather (theta_prev columns staged in smem)
   float lr;
   float mu;
+  // variants (fgd_outer_step_ex): Mix2 only inside column ranges; momentum averaged first
+  int n_ranges;                          // 0 = Mix2 on every column
+  int avg_momentum;                      // 1 = v_m <- mean_n v_n before the update
+  int64_t range_lo[FGD_MAX_RANGES];
+  int64_t range_hi[FGD_MAX_RANGES];
 };
+
+// Is Mix2 applied to the column group starting at `col`?  (Range bounds are multiples of 4
+// columns, so a thread's group is never split.)
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline bool mix2_applies(const StepArgs& a, int64_t col) {
+  if (a.n_ranges == 0) return true;
+  for (int i = 0; i < a.n_ranges; ++i)
+    if (col >= a.range_lo[i] && col < a.range_hi[i]) return true;
+  return false;
+}
 
 }  // namespace fgd
 #endif

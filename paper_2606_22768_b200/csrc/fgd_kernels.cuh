@@ -368,13 +368,19 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
 #pragma unroll
     for (int i = 0; i < VEC; ++i) asum.v[i] = 0.f;
 
+    Pack<VEC> vbar = p_zero<VEC>();              // column mean of the momentum (GlobalM1S option)
+    if (a.avg_momentum) {
+      for (int m = 0; m < K; ++m) vbar = p_add<VEC>(vbar, ld_stream<VEC>(a.momentum + (size_t)m * ld + col));
+      vbar = p_mul<VEC>(vbar, invK);
+    }
+    const bool mixed = mix2_applies(a, col);     // subset option: Mix2 only inside the ranges
     auto finish_row = [&](int m, const Pack<VEC>& gh) {
       const size_t off = (size_t)m * ld + col;
       Pack<VEC> xm;
       if (a.xsrc == XSRC_MATRIX) xm = ld_stream<VEC>(a.x + off);
       else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) xm = gather_row<VEC, BLOCK>(m1, m, tps, tid);
       else xm = xv;
-      const Pack<VEC> v = ld_stream<VEC>(a.momentum + off);
+      const Pack<VEC> v = a.avg_momentum ? vbar : ld_stream<VEC>(a.momentum + off);
       Pack<VEC> vn, tn;
 #pragma unroll
       for (int i = 0; i < VEC; ++i) {
@@ -388,7 +394,10 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
       else if (want_cd) SCol<VEC>::st(avs, m * BLOCK + tid, tn);
     };
 
-    if constexpr (DENSE2) {
+    if (!mixed) {                                 // identity Mix2 on this column group
+#pragma unroll(KT > 0 ? KT : 2)
+      for (int m = 0; m < K; ++m) finish_row(m, SCol<VEC>::ld(gs, m * BLOCK + tid));
+    } else if constexpr (DENSE2) {
       dense_rows<KT, VEC, BLOCK, TR::kRegArrays>(K, wts, gs, tid, finish_row);
     } else {
 #pragma unroll(KT > 0 ? KT : 2)

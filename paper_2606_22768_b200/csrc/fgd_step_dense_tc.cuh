@@ -248,6 +248,14 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       float v[K];
 #pragma unroll
       for (int m = 0; m < K; ++m) v[m] = C[m * T + tid];
+      if (a.avg_momentum) {                        // GlobalM1S option: v_m <- mean_n v_n
+        float vs = 0.f;
+#pragma unroll
+        for (int m = 0; m < K; ++m) vs += v[m];
+        vs *= invK;
+#pragma unroll
+        for (int m = 0; m < K; ++m) v[m] = vs;
+      }
       if (a.xsrc != XSRC_VECTOR) xv = tsum * invK;
       if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier

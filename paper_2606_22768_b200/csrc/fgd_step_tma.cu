@@ -145,7 +145,7 @@ int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix&
 
 // Tensor-core dense step: K = 64, Mix1 given as the averaged row or fused as a mean.
 bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g1) {
-  if (!dense2 || c->K != kTcK || !c->encode_tiled) return false;
+  if (!dense2 || c->K != kTcK || !c->encode_tiled || a.n_ranges != 0) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (!(a.xsrc == XSRC_VECTOR || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;

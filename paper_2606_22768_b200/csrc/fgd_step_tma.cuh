@@ -261,10 +261,22 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
         Pack<VEC> asum = p_zero<VEC>();
         // ---- phase 2: mix, Nesterov step, stream out; theta_new stays in av[] (or in C)
         Pack<VEC> av[KQ];
+        Pack<VEC> vbar = p_zero<VEC>();           // column mean of the momentum (GlobalM1S option)
         if constexpr (REGS) {
 #pragma unroll
           for (int m = 0; m < KQ; ++m) av[m] = SCol<VEC>::ld(C, m * TPB + t);   // momentum, all rows
+          if (a.avg_momentum) {
+#pragma unroll
+            for (int m = 0; m < KQ; ++m) vbar = p_add<VEC>(vbar, av[m]);
+            vbar = p_mul<VEC>(vbar, invK);
+#pragma unroll
+            for (int m = 0; m < KQ; ++m) av[m] = vbar;
+          }
+        } else if (a.avg_momentum) {
+          for (int m = 0; m < K; ++m) vbar = p_add<VEC>(vbar, SCol<VEC>::ld(C, m * TPB + t));
+          vbar = p_mul<VEC>(vbar, invK);
         }
+        const bool mixed = mix2_applies(a, col);   // subset option: Mix2 only inside the ranges
         float* const mom_col = a.momentum + col;
         float* const new_col = a.theta_new + col;
         auto finish_row = [&](int m, const Pack<VEC>& gh) {
@@ -280,7 +292,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           }
           Pack<VEC> v;
           if constexpr (REGS) v = av[m];
-          else v = SCol<VEC>::ld(C, m * TPB + t);
+          else v = a.avg_momentum ? vbar : SCol<VEC>::ld(C, m * TPB + t);
           const Pack<VEC> vn = p_fma<VEC>(v, mu, gh);                       // v' = mu v + ghat
           const Pack<VEC> tn = p_fma<VEC>(p_fma<VEC>(vn, mu, gh), -lr, xm);   // x - lr (ghat + mu v')
           asum = p_add<VEC>(asum, tn);
@@ -297,7 +309,10 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           if constexpr (REGS) av[m] = tn;
           else if (want_cd) SCol<VEC>::st(C, m * TPB + t, tn);
         };
-        if constexpr (DENSE2) {
+        if (!mixed) {                               // identity Mix2 on this column group
+#pragma unroll(KT > 0 ? KT : 2)
+          for (int m = 0; m < K; ++m) finish_row(m, SCol<VEC>::ld(B, m * TPB + t));
+        } else if constexpr (DENSE2) {
           dense_rows<KT, VEC, TPB, (KT > 0 && KT <= 16)>(K, wts, B, t, finish_row);
         } else {
 #pragma unroll(KT > 0 ? KT : 2)

@@ -17,7 +17,7 @@ from typing import Optional
 import torch
 
 from . import (FGD_MIX_IDENTITY, FGD_MIX_MEAN, Context, MixDesc, fgd_consensus_distance, fgd_mix,
-               fgd_outer_step)
+               fgd_outer_step_ex)
 
 
 class OuterRound:
@@ -53,21 +53,24 @@ class OuterRound:
 
     # ---- blocking part: wait for Mix1, then the fused outer step ---------------------------
     def step(self, mix2: MixDesc, theta_local, theta_prev, momentum, theta_new, lr: float = 0.7,
-             mu: float = 0.9, mix1_fused: Optional[MixDesc] = None, want_cd: bool = True) -> None:
+             mu: float = 0.9, mix1_fused: Optional[MixDesc] = None, want_cd: bool = True,
+             mix2_ranges=None, average_momentum: bool = False) -> None:
         """Fused outer step on the current stream.  Uses the pending side-stream Mix1 result,
-        or computes Mix1 inside the kernel when ``mix1_fused`` is given."""
+        or computes Mix1 inside the kernel when ``mix1_fused`` is given.  ``mix2_ranges`` (column
+        ranges Mix2 is restricted to) and ``average_momentum`` select the paper's "-subset" and
+        GlobalM1S variants."""
         cd = self.cd_sumsq if want_cd else None
         if mix1_fused is not None:
-            fgd_outer_step(self.ctx, mix2, mix1_fused, None, False, theta_local, theta_prev, momentum,
-                           theta_new, lr, mu, cd)
+            fgd_outer_step_ex(self.ctx, mix2, mix1_fused, None, False, theta_local, theta_prev, momentum,
+                              theta_new, lr, mu, cd, mix2_ranges, average_momentum)
             return
         if self._pending is None:
             raise RuntimeError("no Mix1 in flight: call launch_mix1() first or pass mix1_fused")
         ev, x, is_vec = self._pending
         self._pending = None
         torch.cuda.current_stream(self.device).wait_event(ev)
-        fgd_outer_step(self.ctx, mix2, None, x, is_vec, theta_local, theta_prev, momentum, theta_new,
-                       lr, mu, cd)
+        fgd_outer_step_ex(self.ctx, mix2, None, x, is_vec, theta_local, theta_prev, momentum, theta_new,
+                          lr, mu, cd, mix2_ranges, average_momentum)
         # the side stream may not overwrite x for the next round before this kernel has read it
         self.side.wait_event(torch.cuda.current_stream(self.device).record_event())
 

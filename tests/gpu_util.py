@@ -93,10 +93,12 @@ class Scenario:
     compares theta_new, momentum and the consensus sums after every round."""
 
     def __init__(self, K, P, mix1, mix2, *, ld=None, seed=0, sigmas=1e-3, worker_std=0.0, mode="factored",
-                 in_place=True, lr=0.7, mu=0.9, v0_std=0.0, path=fgd.FGD_PATH_AUTO):
+                 in_place=True, lr=0.7, mu=0.9, v0_std=0.0, path=fgd.FGD_PATH_AUTO,
+                 mix2_ranges=None, average_momentum=False):
         self.K, self.P, self.ld = K, P, P if ld is None else ld
         self.mix1, self.mix2, self.seed, self.mode, self.in_place = mix1, mix2, seed, mode, in_place
         self.lr, self.mu = lr, mu
+        self.mix2_ranges, self.average_momentum = mix2_ranges, average_momentum
         self.sigmas = np.broadcast_to(np.asarray(sigmas, dtype=np.float32), (K,)).copy()
         th0 = gen.theta0(seed, K, P, 0.02, worker_std)
         v0 = (gen.scaled_normal(seed, gen.TENSOR_MOMENTUM, 0, K, P, v0_std) if v0_std > 0
@@ -123,11 +125,16 @@ class Scenario:
             loc32 = th_prev32 + drift
             self.g_loc.copy_(torch.from_numpy(loc32))
             self.drv.step(m2_desc, self.full_loc, self.full_prev, self.full_v, self.full_new, self.lr, self.mu,
-                          mix1_fused=m1_desc if fused else None, want_cd=True)
+                          mix1_fused=m1_desc if fused else None, want_cd=True,
+                          mix2_ranges=self.mix2_ranges, average_momentum=self.average_momentum)
             torch.cuda.synchronize()
             # oracle, free running: its own float64 state plus the shared drift
             o_loc = self.o_theta + drift.astype(np.float64)
-            self.o_theta, self.o_v = oracle.outer_round(W1, W2, self.o_theta, o_loc, self.o_v, self.lr, self.mu)
+            if self.mix2_ranges is None and not self.average_momentum:
+                self.o_theta, self.o_v = oracle.outer_round(W1, W2, self.o_theta, o_loc, self.o_v, self.lr, self.mu)
+            else:
+                self.o_theta, self.o_v = oracle.outer_round_ex(W1, W2, self.o_theta, o_loc, self.o_v, self.lr, self.mu,
+                                                               self.mix2_ranges, self.average_momentum)
             assert_param_close(self.g_new, self.o_theta, f"theta_new round {r}")
             assert_param_close(self.g_v, self.o_v, f"momentum round {r}")
             assert_cd_close(self.drv.cd_sumsq, oracle.consensus_sumsq(self.o_theta), P, f"cd_sumsq round {r}")

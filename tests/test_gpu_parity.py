@@ -271,6 +271,55 @@ def test_nonzero_initial_momentum_and_odd_K():
     Scenario(32, 12346, ("mean",), ("hypercube", 0.05), seed=6, v0_std=1e-3).run(3)
 
 
+# ------------------------------------------------------------------ the paper's variants: -subset and GlobalM1S
+def _subset(P):
+    """About 43 % of the columns in three blocks (embeddings, LM head, first layers), on 4-column bounds."""
+    a, b, c = int(0.18 * P) // 4 * 4, int(0.55 * P) // 4 * 4, int(0.80 * P) // 4 * 4
+    return [(0, a), (b, c - (c - b) // 3 // 4 * 4), (c, P)]
+
+
+VARIANTS = [
+    # name, K, P, mix1, mix2, subset?, average momentum?
+    ("GlobalM1LocalM2-subset", 8, 40004, ("mean",), ("matching",), True, False),
+    ("GlobalM1S", 8, 30000, ("mean",), ("identity",), False, True),
+    ("GlobalM1SLocalM2", 16, 30001, ("mean",), ("matching",), False, True),
+    ("GlobalM1SLocalM2-subset", 16, 50000, ("mean",), ("matching",), True, True),
+    ("ring-subset-runtimeK", 6, 9000, ("mean",), ("ring",), True, True),
+    ("dense-subset", 64, 6000, ("mean",), ("dense", SINK64), True, False),
+    ("dense-GlobalM1S", 64, 5000, ("mean",), ("dense", SINK64), False, True),
+    ("dense16-subset", 16, 8000, ("ring",), ("dense", gen.sinkhorn_W(1, 16)), True, False),
+]
+
+
+@pytest.mark.parametrize("name,K,P,mix1,mix2,subset,avg", VARIANTS, ids=[v[0] for v in VARIANTS])
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("mode", ["factored", "fused"])
+def test_paper_variants(name, K, P, mix1, mix2, subset, avg, path, mode):
+    ld = P + (4 - P % 4) % 4
+    Scenario(K, P, mix1, mix2, ld=ld, seed=4, v0_std=1e-3, worker_std=5e-4, mode=mode, path=path,
+             mix2_ranges=_subset(P) if subset else None, average_momentum=avg).run(3)
+
+
+def test_variant_argument_errors():
+    K, P = 4, 1024
+    ctx = fgd.Context(K, P)
+    a = torch.zeros((K, P), device="cuda")
+    b, c, d = torch.zeros_like(a), torch.zeros_like(a), torch.zeros_like(a)
+    ring, mean = fgd.MixDesc.ring(K), fgd.MixDesc.mean(K)
+    with pytest.raises(fgd.FgdError) as e:    # range bounds must be multiples of 4 columns
+        fgd.fgd_outer_step_ex(ctx, ring, mean, None, False, b, a, c, d, mix2_ranges=[(2, 8)])
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:    # beyond P
+        fgd.fgd_outer_step_ex(ctx, ring, mean, None, False, b, a, c, d, mix2_ranges=[(0, P + 4)])
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:    # too many ranges
+        fgd.fgd_outer_step_ex(ctx, ring, mean, None, False, b, a, c, d, mix2_ranges=[(4 * i, 4 * i + 4) for i in range(9)])
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:    # momentum averaging belongs to a global Mix1
+        fgd.fgd_outer_step_ex(ctx, ring, ring, None, False, b, a, c, d, average_momentum=True)
+    assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------------ determinism, errors
 def test_outer_step_is_bitwise_deterministic():
     K, P = 16, 200000
