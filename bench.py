@@ -66,6 +66,8 @@ def parse_args():
     ap.add_argument("--subset-frac", type=float, default=0.0,
                     help="variant: restrict Mix2 to about this fraction of the columns (three blocks)")
     ap.add_argument("--average-momentum", action="store_true", help="variant: GlobalM1S (needs Mix1 = mean)")
+    ap.add_argument("--kernels", action="store_true",
+                    help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -269,6 +271,11 @@ def run_ours(args):
         if ev_pair is not None:
             ev_pair[1].record(main)
 
+    if args.kernels:
+        if rank == 0:
+            print(json.dumps(kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, measured_peak())), flush=True)
+        return
+
     for r in range(warmup):
         one_round(r)
     torch.cuda.synchronize()
@@ -337,6 +344,50 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, peak, reps=10):
+    """Each C-ABI kernel of this config timed alone (CUDA events, mean of `reps` after 3 warm-ups),
+    with its algorithmic bytes: GB/s and fraction of the measured HBM peak."""
+    K, P = cfg["K"], cfg["P"]
+    dev = theta.device
+    ctx = drv.ctx
+    scratch = torch.empty_like(theta)
+    xvec = torch.empty(P, dtype=torch.float32, device=dev)
+    cd = torch.zeros(K, dtype=torch.float64, device=dev)
+    m1 = mix_desc(fgd, cfg["mix1"], cfg, 0, seed, 1, dense_W)
+    m2 = mix_desc(fgd, cfg["mix2"], cfg, 0, seed, 2, dense_W)
+    mean = fgd.MixDesc.mean(K)
+    fgd.fgd_mix(ctx, mean, theta, xvec, out_is_vector=True)
+    WP = K * P
+    cases = {
+        "fgd_outer_grad": (lambda: fgd.fgd_outer_grad(ctx, theta, local, scratch), 12 * WP),
+        "fgd_mix mean -> [P]": (lambda: fgd.fgd_mix(ctx, mean, theta, xvec, out_is_vector=True), 4 * WP + 4 * P),
+        "fgd_mix Mix2 kind -> [K,P]": (lambda: fgd.fgd_mix(ctx, m2, theta, scratch), 8 * WP),
+        "fgd_consensus_distance": (lambda: fgd.fgd_consensus_distance(ctx, theta, cd), 4 * WP),
+        "fgd_outer_step x=[P], with consensus": (lambda: fgd.fgd_outer_step(ctx, m2, None, xvec, True, local, theta, mom, theta, 0.7, 0.9, cd), 20 * WP + 4 * P),
+        "fgd_outer_step x=[P], no consensus": (lambda: fgd.fgd_outer_step(ctx, m2, None, xvec, True, local, theta, mom, theta, 0.7, 0.9, None), 20 * WP + 4 * P),
+        "fgd_outer_step Mix1 mean fused": (lambda: fgd.fgd_outer_step(ctx, m2, mean, None, False, local, theta, mom, theta, 0.7, 0.9, cd), 20 * WP),
+        "fgd_outer_step x=[K,P]": (lambda: fgd.fgd_outer_step(ctx, m2, None, scratch, False, local, theta, mom, theta, 0.7, 0.9, cd), 24 * WP),
+    }
+    if cfg["mix1"][0] not in ("mean", "dense"):
+        cases["fgd_outer_step Mix1 gossip fused"] = (lambda: fgd.fgd_outer_step(ctx, m2, m1, None, False, local, theta, mom, theta, 0.7, 0.9, cd), 20 * WP)
+    out = {"workload": cfg["name"], "peak_gbs": peak[0], "peak_kind": peak[1], "kernels": {}}
+    for name, (fn, nbytes) in cases.items():
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out["kernels"][name] = {"ms": round(ms, 4), "algorithmic_gb": round(nbytes / 1e9, 2), "gbs": round(gbs, 1),
+                                "frac": round(gbs / peak[0], 3)}
+    return out
 
 
 def copy_bandwidth(torch, dev, n=1 << 30, reps=10):
