@@ -68,6 +68,8 @@ def parse_args():
     ap.add_argument("--average-momentum", action="store_true", help="variant: GlobalM1S (needs Mix1 = mean)")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
+    ap.add_argument("--js", action="store_true",
+                    help="instead of the round: time the JS functional-disagreement metric on synthetic logits")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -232,6 +234,10 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.js:
+        if rank == 0:
+            print(json.dumps(js_table(torch, fgd, dev, measured_peak())), flush=True)
+        return
     cfg = dict(CONFIGS[args.config])
     if args.cols:
         cfg["P"] = args.cols
@@ -388,6 +394,34 @@ def kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, peak, r
         out["kernels"][name] = {"ms": round(ms, 4), "algorithmic_gb": round(nbytes / 1e9, 2), "gbs": round(gbs, 1),
                                 "frac": round(gbs / peak[0], 3)}
     return out
+
+
+def js_table(torch, fgd, dev, peak, K=8, U=4096, V=128256, k=100, reps=5):
+    """JS metric on synthetic logits shaped like a Llama-3 vocabulary: K workers, U token positions.
+    Algorithmic bytes = one read of the averaged model's logits (U V 4) plus the gathered entries."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(0)
+    avg = torch.randn((U, V), device=dev, generator=g) * 2.0
+    work = torch.empty((K, U, V), device=dev)
+    for m in range(K):
+        work[m] = avg + 0.3 * torch.randn((U, V), device=dev, generator=g)
+    idx = torch.empty((U, k), dtype=torch.int32, device=dev)
+    d = torch.empty((K, U), dtype=torch.float64, device=dev)
+    cdw = torch.empty(K, dtype=torch.float64, device=dev)
+    for _ in range(2):
+        fgd.fgd_js_distance(work, avg, idx, d, cdw, top_k=k)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fgd.fgd_js_distance(work, avg, idx, d, cdw, top_k=k)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    nbytes = U * V * 4 + (K + 1) * U * k * 32      # gathers move one 32-byte sector per entry
+    return {"metric": "js_token_positions_per_s", "value": U / (ms * 1e-3), "ms": ms, "K": K, "U": U, "V": V, "top_k": k,
+            "algorithmic_gb": nbytes / 1e9, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak[0],
+            "cd_js": float(cdw.mean())}
 
 
 def copy_bandwidth(torch, dev, n=1 << 30, reps=10):

@@ -177,6 +177,20 @@ int fgd_outer_step_ex(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc
  * fgd_cd_finalize. */
 int fgd_consensus_distance(fgd_ctx* ctx, const float* theta, double* cd_sumsq, void* stream);
 
+/* JS functional disagreement (App. D.2): for every token position u the normalised
+ * Jensen-Shannon distance sqrt(JS / ln 2) between worker m's softmax distribution and the
+ * parameter-averaged model's, computed in float64 in the log domain on the top_k tokens of the
+ * averaged model only (the paper uses 100; both distributions are restricted to those tokens
+ * and renormalised; ties at the cut go to the lower token index).  CD_JS is the mean of d_js.
+ *   worker_logits device [K, U, V] fp32, avg_logits device [U, V] fp32 (the model forward that
+ *   produces them is not part of this library);
+ *   top_idx  device [U, top_k] int32 out: the selected tokens of each position, ascending;
+ *   d_js     device [K, U] doubles out;  cd_worker device [K] doubles out: mean over u.
+ * 1 <= top_k <= min(256, V).  Needs no context and allocates nothing. */
+int fgd_js_distance(int device, int K, int64_t U, int64_t V, int top_k, const float* worker_logits,
+                    const float* avg_logits, int32_t* top_idx, double* d_js, double* cd_worker,
+                    void* stream);
+
 /* (No counterpart in the paper: a packaging variant of fgd_consensus_distance.)
  * Same result as fgd_consensus_distance, for callers that cannot allocate GPU memory and so
  * cannot create a context: it needs no fgd_ctx and calls no cudaMalloc / cudaFree or any other

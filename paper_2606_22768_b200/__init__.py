@@ -71,6 +71,7 @@ def _load():
         "fgd_outer_step_ex": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp, vp]),
         "fgd_consensus_distance": (i32, [vp, vp, vp, vp]),
         "fgd_consensus_distance_noalloc": (i32, [i32, i32, i64, i64, vp, vp, vp]),
+        "fgd_js_distance": (i32, [i32, i32, i64, i64, i32, vp, vp, vp, vp, vp, vp]),
         "fgd_topo_ring": (i32, [i32, vp, vp, vp]),
         "fgd_topo_onepeer_xor": (i32, [i32, i64, vp, vp, vp]),
         "fgd_topo_hypercube": (i32, [i32, vp, vp, vp]),
@@ -339,5 +340,19 @@ def fgd_consensus_distance_noalloc(device: int, K: int, P: int, ld: int, theta, 
     rc = _lib.fgd_consensus_distance_noalloc(int(device), int(K), int(P), int(ld),
                                              _dev_ptr(theta, "theta", "torch.float32"),
                                              _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), _stream(stream))
+    if rc != 0:
+        raise FgdError(rc, fgd_last_error(None))
+
+
+def fgd_js_distance(worker_logits, avg_logits, top_idx, d_js, cd_worker, top_k: int = 100, device: int = 0,
+                    stream=None) -> None:
+    """JS functional disagreement of [K, U, V] worker logits against [U, V] averaged-model logits
+    on the averaged model's top_k tokens; fills top_idx [U, top_k], d_js [K, U], cd_worker [K]."""
+    K, U, V = worker_logits.shape
+    rc = _lib.fgd_js_distance(int(device), int(K), int(U), int(V), int(top_k),
+                              _dev_ptr(worker_logits, "worker_logits", "torch.float32"),
+                              _dev_ptr(avg_logits, "avg_logits", "torch.float32"),
+                              _dev_ptr(top_idx, "top_idx", "torch.int32"), _dev_ptr(d_js, "d_js", "torch.float64"),
+                              _dev_ptr(cd_worker, "cd_worker", "torch.float64"), _stream(stream))
     if rc != 0:
         raise FgdError(rc, fgd_last_error(None))

@@ -54,3 +54,43 @@ def test_top_tokens_and_truncated_metric():
     # identical workers and average: zero disagreement
     _, d0, cd0 = ojs.cd_js(np.stack([avg, avg]), avg, k)
     assert cd0 == 0.0 and d0.max() == 0.0
+
+
+# ------------------------------------------------------------------ GPU parity
+@pytest.mark.gpu
+@pytest.mark.parametrize("K,U,V,k", [(4, 64, 32000, 100), (8, 33, 5001, 100), (2, 7, 100, 100), (3, 5, 70000, 37), (1, 1, 256, 1)])
+def test_js_distance_gpu(K, U, V, k):
+    import torch
+    import paper_2606_22768_b200 as fgd
+    work, avg = _logits(K, U, V, seed=3)
+    if V == 5001:                      # force ties at the cut: many equal logits in the averaged model
+        avg[:, ::7] = 1.25
+    w = torch.from_numpy(work).cuda()
+    a = torch.from_numpy(avg).cuda()
+    idx = torch.full((U, k), -1, dtype=torch.int32, device="cuda")
+    d = torch.full((K, U), -1.0, dtype=torch.float64, device="cuda")
+    cdw = torch.zeros(K, dtype=torch.float64, device="cuda")
+    fgd.fgd_js_distance(w, a, idx, d, cdw, top_k=k)
+    torch.cuda.synchronize()
+    ref_idx, ref_d, ref_cd = ojs.cd_js(work, avg, k)
+    assert np.array_equal(idx.cpu().numpy().astype(np.int64), ref_idx), "selected tokens must match exactly"
+    np.testing.assert_allclose(d.cpu().numpy(), ref_d, rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(cdw.cpu().numpy(), ref_d.mean(axis=1), rtol=1e-10, atol=1e-13)
+    assert float(cdw.mean()) == pytest.approx(ref_cd, rel=1e-10, abs=1e-13)
+    # deterministic
+    d2 = torch.zeros_like(d)
+    fgd.fgd_js_distance(w, a, idx, d2, cdw, top_k=k)
+    torch.cuda.synchronize()
+    assert torch.equal(d, d2)
+
+
+@pytest.mark.gpu
+def test_js_distance_argument_errors():
+    import torch
+    import paper_2606_22768_b200 as fgd
+    w = torch.zeros((2, 3, 50), device="cuda"); a = torch.zeros((3, 50), device="cuda")
+    idx = torch.zeros((3, 100), dtype=torch.int32, device="cuda")
+    d = torch.zeros((2, 3), dtype=torch.float64, device="cuda"); c = torch.zeros(2, dtype=torch.float64, device="cuda")
+    with pytest.raises(fgd.FgdError) as e:
+        fgd.fgd_js_distance(w, a, idx, d, c, top_k=100)    # more tokens than the vocabulary has
+    assert e.value.status == fgd.FGD_ERR_INVALID_ARG
