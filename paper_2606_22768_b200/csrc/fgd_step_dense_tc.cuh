@@ -261,6 +261,10 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }
+      // the MMA has consumed the operands and this column's momentum is in registers: the stage can
+      // be refilled while the epilogue below runs from registers and tensor memory
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float gh[K];
       tmem_ld_64(tmem_base + ((uint32_t)(warp * 32) << 16), gh);
@@ -287,8 +291,6 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           }
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(smem_u32(&bars[STAGES + s]));
     }
   }
 
