@@ -140,7 +140,8 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
 
   return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
-    size_t smem = sizeof(float) * (size_t)K * kBlock * VECc;
+    // the averaging path keeps everything in registers: no private columns, more CTAs per SM
+    size_t smem = desc->kind == FGD_MIX_MEAN ? 0 : sizeof(float) * (size_t)K * kBlock * VECc;
     int grid = 0;
     if (dense) {
       smem += sizeof(float) * (size_t)K * K;

@@ -465,21 +465,22 @@ __global__ void __launch_bounds__(BLOCK) mix_kernel(const MixArgs a, const MX mx
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t col = (tile * BLOCK + tid) * VEC;
     if (col >= P) continue;
-    Pack<VEC> sum;
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) sum.v[i] = 0.f;
     bool is_mean = false;
     if constexpr (!DENSE) is_mean = (mx.kind == KMIX_MEAN);
-#pragma unroll(KT > 0 ? KT : 4)
-    for (int m = 0; m < K; ++m) {
-      const Pack<VEC> t = ld_stream<VEC>(a.in + (size_t)m * ld + col);
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) sum.v[i] += t.v[i];
-      if (!is_mean) SCol<VEC>::st(cs, m * BLOCK + tid, t);
-    }
     if (is_mean) {
+      // pure load-and-add: nothing between the K loads, so they are all in flight together
+      Pack<VEC> sum = p_zero<VEC>();
+      if constexpr (KT > 0) {
+        Pack<VEC> t[KT];
 #pragma unroll
-      for (int i = 0; i < VEC; ++i) sum.v[i] *= invK;
+        for (int m = 0; m < KT; ++m) t[m] = ld_stream<VEC>(a.in + (size_t)m * ld + col);
+#pragma unroll
+        for (int m = 0; m < KT; ++m) sum = p_add<VEC>(sum, t[m]);
+      } else {
+#pragma unroll 4
+        for (int m = 0; m < K; ++m) sum = p_add<VEC>(sum, ld_stream<VEC>(a.in + (size_t)m * ld + col));
+      }
+      sum = p_mul<VEC>(sum, invK);
       if (a.out_is_vector) {
         st_stream<VEC>(a.out + col, sum);
       } else {
@@ -487,6 +488,17 @@ __global__ void __launch_bounds__(BLOCK) mix_kernel(const MixArgs a, const MX mx
         for (int m = 0; m < K; ++m) st_stream<VEC>(a.out + (size_t)m * ld + col, sum);
       }
       continue;
+    }
+    // all rows of the column group into the private column (loads first, then the stores)
+    if constexpr (KT > 0) {
+      Pack<VEC> t[KT];
+#pragma unroll
+      for (int m = 0; m < KT; ++m) t[m] = ld_stream<VEC>(a.in + (size_t)m * ld + col);
+#pragma unroll
+      for (int m = 0; m < KT; ++m) SCol<VEC>::st(cs, m * BLOCK + tid, t[m]);
+    } else {
+#pragma unroll 4
+      for (int m = 0; m < K; ++m) SCol<VEC>::st(cs, m * BLOCK + tid, ld_stream<VEC>(a.in + (size_t)m * ld + col));
     }
     if constexpr (DENSE) {
       dense_rows<KT, VEC, BLOCK, false>(K, wts, cs, tid, [&](int m, const Pack<VEC>& r) {
