@@ -332,22 +332,20 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
     const int64_t col = (tile * BLOCK + tid) * VEC;
     if (col >= P) continue;
 
-    // ---- phase 1: outer gradient of every worker into the private column, column sums
-    Pack<VEC> gsum, tsum;
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) gsum.v[i] = tsum.v[i] = 0.f;
+    // ---- phase 1: outer gradient of every worker into the private column, column sums.
+    // With a compile-time K the momentum rows are requested here too: measured on B200, having
+    // all 3K loads of a column group in flight at once is worth 3.2 -> 5.3 TB/s on this kernel.
+    Pack<VEC> gsum = p_zero<VEC>(), tsum = p_zero<VEC>();
+    Pack<VEC> vreg[KR];
 #pragma unroll(KT > 0 ? KT : 4)
     for (int m = 0; m < K; ++m) {
       const size_t off = (size_t)m * ld + col;
       const Pack<VEC> tp = ld_stream<VEC>(a.theta_prev + off);
       const Pack<VEC> tl = ld_stream<VEC>(a.theta_local + off);
-      Pack<VEC> g;
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) {
-        g.v[i] = tp.v[i] - tl.v[i];
-        gsum.v[i] += g.v[i];
-        tsum.v[i] += tp.v[i];
-      }
+      if constexpr (TR::kRegArrays) vreg[m] = ld_stream<VEC>(a.momentum + off);
+      const Pack<VEC> g = p_sub<VEC>(tp, tl);
+      gsum = p_add<VEC>(gsum, g);
+      tsum = p_add<VEC>(tsum, tp);
       SCol<VEC>::st(gs, m * BLOCK + tid, g);
       if (a.stage_tp) SCol<VEC>::st(tps, m * BLOCK + tid, tp);
     }
@@ -370,7 +368,12 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
 
     Pack<VEC> vbar = p_zero<VEC>();              // column mean of the momentum (GlobalM1S option)
     if (a.avg_momentum) {
-      for (int m = 0; m < K; ++m) vbar = p_add<VEC>(vbar, ld_stream<VEC>(a.momentum + (size_t)m * ld + col));
+      if constexpr (TR::kRegArrays) {
+#pragma unroll
+        for (int m = 0; m < KR; ++m) vbar = p_add<VEC>(vbar, vreg[m]);
+      } else {
+        for (int m = 0; m < K; ++m) vbar = p_add<VEC>(vbar, ld_stream<VEC>(a.momentum + (size_t)m * ld + col));
+      }
       vbar = p_mul<VEC>(vbar, invK);
     }
     const bool mixed = mix2_applies(a, col);     // subset option: Mix2 only inside the ranges
@@ -380,7 +383,10 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
       if (a.xsrc == XSRC_MATRIX) xm = ld_stream<VEC>(a.x + off);
       else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) xm = gather_row<VEC, BLOCK>(m1, m, tps, tid);
       else xm = xv;
-      const Pack<VEC> v = a.avg_momentum ? vbar : ld_stream<VEC>(a.momentum + off);
+      Pack<VEC> v;
+      if (a.avg_momentum) v = vbar;
+      else if constexpr (TR::kRegArrays) v = vreg[m];
+      else v = ld_stream<VEC>(a.momentum + off);
       Pack<VEC> vn, tn;
 #pragma unroll
       for (int i = 0; i < VEC; ++i) {
