@@ -82,29 +82,47 @@ __device__ __forceinline__ void tmem_ld_64(uint32_t taddr, float (&r)[64]) {
 }
 
 constexpr int kTcK = 64;            // workers (MMA K and N dimensions)
-constexpr int kTcCols = 128;        // columns per tile (MMA M dimension) = consumer threads
+constexpr int kTcCols = 128;        // columns per tile (MMA M dimension)
+constexpr int kTcHalf = kTcK / 2;   // workers per consumer thread: two threads share a column
+constexpr int kTcConsumers = 2 * kTcCols;
 constexpr int kTcStages = 2;
 constexpr int kTcTmemCols = 64;     // fp32 accumulator columns (= K), a power of two >= 32
 constexpr uint32_t kTcBox = kTcK * kTcCols * sizeof(float);   // 32 KB: one tensor of a stage
 constexpr uint32_t kTcWBytes = kTcK * kTcK * sizeof(float);   // 16 KB: one split of W
-// dynamic shared memory: 1 KB alignment slack + stages + W_hi + W_lo
-constexpr size_t kTcSmem = 1024 + (size_t)kTcStages * 3 * kTcBox + 2 * kTcWBytes;
+// dynamic shared memory: alignment slack + stages + W_hi + W_lo
+constexpr size_t kTcSmem = 128 + (size_t)kTcStages * 3 * kTcBox + 2 * kTcWBytes;
 
-__global__ void __launch_bounds__(kTcCols + 32)
+// 32 lanes x 32 bit x 32 columns: thread i of the warp receives 32 consecutive columns of lane (base + i).
+__device__ __forceinline__ void tmem_ld_32(uint32_t taddr, float (&r)[32]) {
+  uint32_t* u = reinterpret_cast<uint32_t*>(r);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+        "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+        "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                            const __grid_constant__ CUtensorMap tm_mom) {
-  constexpr int K = kTcK, T = kTcCols, STAGES = kTcStages;
+  constexpr int K = kTcK, T = kTcCols, H = kTcHalf, CONS = kTcConsumers, STAGES = kTcStages;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];   // full[], empty[], mma
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_slot;
+  __shared__ float xchg[2][T];       // the two halves of a column exchange their theta_new sums
 
   const StepArgs& a = ta.s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool want_cd = a.partials != nullptr;
-  // operand regions on 1024-byte boundaries
-  unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* base = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // TMA wants 128-byte alignment
   unsigned char* wb_hi = base + (size_t)STAGES * 3 * kTcBox;
   unsigned char* wb_lo = wb_hi + kTcWBytes;
   const uint32_t mma_bar = smem_u32(&bars[2 * STAGES]);
@@ -116,14 +134,14 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bars[s]), 1);
-      mbar_init(smem_u32(&bars[STAGES + s]), T);
+      mbar_init(smem_u32(&bars[STAGES + s]), CONS);
     }
     mbar_init(mma_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // B operand = W^T as an N x K (m x n) matrix, K-major, no swizzle: 8-row x 16-byte core
   // matrices; core matrices adjacent in K are 128 B apart, adjacent in N 2048 B apart.
-  for (int i = tid; i < K * K; i += T + 32) {
+  for (int i = tid; i < K * K; i += CONS + 32) {
     const int n = i / K, m = i % K;          // m2.Wt[n*K+m] = W[m][n]
     const float w = m2.Wt[i];
     const float hi = to_tf32(w);
@@ -131,7 +149,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     *reinterpret_cast<float*>(wb_hi + off) = hi;
     *reinterpret_cast<float*>(wb_lo + off) = w - hi;
   }
-  if (warp == T / 32) {   // the producer warp owns tensor memory: allocate K accumulator columns
+  if (warp == CONS / 32) {   // the producer warp owns tensor memory: allocate the accumulator columns
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTcTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -141,11 +159,11 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_slot;
 
-  float sacc[K];
+  float sacc[H];
 #pragma unroll
-  for (int m = 0; m < K; ++m) sacc[m] = 0.f;
+  for (int m = 0; m < H; ++m) sacc[m] = 0.f;
 
-  if (warp == T / 32) {
+  if (warp == CONS / 32) {
     // ===================================================== producer (one elected lane)
     if (lane == 0) {
       uint64_t policy;
@@ -173,21 +191,25 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       }
     }
   } else {
-    // ===================================================== consumers: thread t owns column t of the tile
+    // ===================================================== consumers
+    // Two threads per column: thread (c, h) owns column c of the tile and the workers
+    // [32 h, 32 h + 32) -- eight consumer warps instead of four hide the shared-memory, TMEM and
+    // barrier latencies, and 32 instead of 64 values per array keep everything in registers.
+    const int c = tid & (T - 1), h = tid >> 7, r0 = h * H;
     const float invK = 1.0f / (float)K;
     const float lr = a.lr, mu = a.mu;
     const bool need_tsum = a.xsrc == XSRC_FUSED;                      // fused mean Mix1
     // A operand = g^T as an M x K (column x worker) matrix, K-major, no swizzle, same core-matrix
-    // scheme as B: row `tid`, four consecutive workers = one 16-byte core-matrix row, so a
-    // thread's 64 values go out as 16 conflict-free 128-bit stores.
-    const uint32_t op_row = (uint32_t)(tid >> 3) * 2048u + (uint32_t)(tid & 7) * 16u;
+    // scheme as B: row c, four consecutive workers = one 16-byte core-matrix row, so a thread's
+    // 32 values go out as 8 conflict-free 128-bit stores.
+    const uint32_t op_row = (uint32_t)(c >> 3) * 2048u + (uint32_t)(c & 7) * 16u;
     // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
     constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
     int64_t i = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
       const int s = (int)(i % STAGES);
       const uint32_t use = (uint32_t)(i / STAGES);
-      const int64_t col = tile * T + tid;
+      const int64_t col = tile * T + c;
       const bool live = col < P;
       float xv = 0.f;
       if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
@@ -195,38 +217,42 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       float* A = reinterpret_cast<float*>(stage);                 // theta_prev  -> g_lo operand
       float* B = reinterpret_cast<float*>(stage + kTcBox);        // theta_local -> g_hi operand
       float* C = reinterpret_cast<float*>(stage + 2 * kTcBox);    // momentum
-      // ---- phase 1: g for all workers in registers
-      float g[K];
+      // ---- phase 1: g of this thread's workers in registers
+      float g[H];
       float tsum = 0.f;
       const bool got = mbar_wait(smem_u32(&bars[s]), use & 1);
       if (got) {
 #pragma unroll
-        for (int n = 0; n < K; ++n) {
-          const float tp = A[n * T + tid];
-          g[n] = tp - B[n * T + tid];
-          if (need_tsum) tsum += tp;
+        for (int n = 0; n < H; ++n) {
+          const float tp = A[(r0 + n) * T + c];
+          g[n] = tp - B[(r0 + n) * T + c];
+          tsum += tp;
+        }
+        if (need_tsum) {                           // the column mean needs the other half too
+#pragma unroll
+          for (int n = 0; n < H; ++n) tsum += A[((H - r0) + n) * T + c];
         }
       } else {
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }
-      named_bar_sync(1, T);                       // every consumer has read its theta_prev / theta_local
+      named_bar_sync(1, CONS);                    // every consumer has read its theta_prev / theta_local
       if (*(volatile int*)&abort_flag) break;     // uniform: the flag was written before the barrier
       // ---- operands: g_hi over the theta_local box, g_lo over the theta_prev box
 #pragma unroll
-      for (int n = 0; n < K; n += 4) {
+      for (int n = 0; n < H; n += 4) {
         float4 hi, lo;
         hi.x = to_tf32(g[n]);     lo.x = g[n] - hi.x;
         hi.y = to_tf32(g[n + 1]); lo.y = g[n + 1] - hi.y;
         hi.z = to_tf32(g[n + 2]); lo.z = g[n + 2] - hi.z;
         hi.w = to_tf32(g[n + 3]); lo.w = g[n + 3] - hi.w;
-        const uint32_t off = op_row + (uint32_t)(n >> 2) * 128u;
+        const uint32_t off = op_row + (uint32_t)((r0 + n) >> 2) * 128u;
         *reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(B) + off) = hi;
         *reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(A) + off) = lo;
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      named_bar_sync(2, T);                       // operands complete; last tile's TMEM reads are done too
+      named_bar_sync(2, CONS);                    // operands complete; last tile's TMEM reads are done too
       if (tid == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_hi = smem_u32(B), a_lo = smem_u32(A);
@@ -244,37 +270,37 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         }
         umma_commit(mma_bar);
       }
-      // ---- while the tensor core works: this column's momentum from the stage
-      float v[K];
+      // ---- while the tensor core works: this thread's momentum values from the stage
+      float v[H];
 #pragma unroll
-      for (int m = 0; m < K; ++m) v[m] = C[m * T + tid];
-      if (a.avg_momentum) {                        // GlobalM1S option: v_m <- mean_n v_n
+      for (int m = 0; m < H; ++m) v[m] = C[(r0 + m) * T + c];
+      if (a.avg_momentum) {                        // GlobalM1S option: v_m <- mean_n v_n (all 64 workers)
         float vs = 0.f;
 #pragma unroll
-        for (int m = 0; m < K; ++m) vs += v[m];
+        for (int m = 0; m < H; ++m) vs += v[m] + C[((H - r0) + m) * T + c];
         vs *= invK;
 #pragma unroll
-        for (int m = 0; m < K; ++m) v[m] = vs;
+        for (int m = 0; m < H; ++m) v[m] = vs;
       }
       if (a.xsrc != XSRC_VECTOR) xv = tsum * invK;
       if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }
-      // the MMA has consumed the operands and this column's momentum is in registers: the stage can
+      // the MMA has consumed the operands and this thread's momentum is in registers: the stage can
       // be refilled while the epilogue below runs from registers and tensor memory
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float gh[K];
-      tmem_ld_64(tmem_base + ((uint32_t)(warp * 32) << 16), gh);
-      // ---- phase 2: Nesterov step for every worker of this column, stream out
+      float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
+      tmem_ld_32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
+      // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
       float asum = 0.f;
       if (live) {
-        float* const mom_col = a.momentum + col;
-        float* const new_col = a.theta_new + col;
+        float* const mom_col = a.momentum + (size_t)r0 * ld + col;
+        float* const new_col = a.theta_new + (size_t)r0 * ld + col;
 #pragma unroll
-        for (int m = 0; m < K; ++m) {
+        for (int m = 0; m < H; ++m) {
           const float vn = fmaf(mu, v[m], gh[m]);
           const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xv);
           __stcs(mom_col + (size_t)m * ld, vn);
@@ -282,10 +308,14 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           v[m] = tn;
           asum += tn;
         }
-        if (want_cd) {
-          const float mean = asum * invK;
+      }
+      if (want_cd) {                               // column mean over both halves, then squared deviations
+        xchg[h][c] = asum;
+        named_bar_sync(3, CONS);
+        const float mean = (asum + xchg[h ^ 1][c]) * invK;
+        if (live) {
 #pragma unroll
-          for (int m = 0; m < K; ++m) {
+          for (int m = 0; m < H; ++m) {
             const float d = v[m] - mean;
             sacc[m] = fmaf(d, d, sacc[m]);
           }
@@ -297,26 +327,27 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   // ---- wrap-up: tensor memory back, consensus partial sums (stage memory is free now)
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == T / 32) {
+  if (warp == CONS / 32) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTcTmemCols) : "memory");
   }
   if (want_cd) {
-    double* red = reinterpret_cast<double*>(base);    // [T/32][K]
-    if (warp < T / 32) {
+    double* red = reinterpret_cast<double*>(base);    // [CONS/32][H]: warps 0-3 hold workers 0-31, warps 4-7 workers 32-63
+    if (warp < CONS / 32) {
 #pragma unroll
-      for (int m = 0; m < K; ++m) {
+      for (int m = 0; m < H; ++m) {
         double d = (double)sacc[m];
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
-        if (lane == 0) red[warp * K + m] = d;
+        if (lane == 0) red[warp * H + m] = d;
       }
     }
     __syncthreads();
     if (tid < K) {
+      const int hh = tid / H, mm = tid % H;
       double d = 0.0;
 #pragma unroll
-      for (int w = 0; w < T / 32; ++w) d += red[w * K + tid];
+      for (int w = 0; w < T / 32; ++w) d += red[(hh * (T / 32) + w) * H + mm];
       a.partials[(size_t)blockIdx.x * K + tid] = d;
     }
   }

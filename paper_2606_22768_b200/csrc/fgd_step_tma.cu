@@ -149,7 +149,7 @@ bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, const Gat
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (!(a.xsrc == XSRC_VECTOR || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
-  return (size_t)c->max_smem_optin >= kTcSmem + 1024;
+  return (size_t)c->max_smem_optin >= kTcSmem + 2048;
 }
 
 int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, const GatherMix& g1, cudaStream_t st,
@@ -166,8 +166,8 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
   int grid = 0;
   auto kern = outer_step_dense_tc_kernel;
-  if (int r = persistent_grid(c, kern, kTcCols + 32, kTcSmem, ntiles, &grid)) return r;
-  kern<<<grid, kTcCols + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
+  kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
   *grid_out = grid;
   return check_launch(c, "outer_step_dense_tc_kernel");
 }
