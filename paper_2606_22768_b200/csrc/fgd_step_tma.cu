@@ -105,29 +105,34 @@ int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix&
   // (identity 0, one-peer / matching 1, ring 2, hypercube of 16 workers 4); else read at run time
   int d2t = -1;
   if (!dense2 && g2.kind == KMIX_GATHER && (g2.D == 0 || g2.D == 1 || g2.D == 2 || g2.D == 4)) d2t = g2.D;
-  auto go = [&]<int KTc, int VECc, int Cc, int D2c>() -> int {
+  // a fused gather Mix1 with the same neighbour count as Mix2 (both mixes on one topology, as in
+  // the paper's LocalM1M2) also gets a static gather
+  const bool same_d1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER && d2t > 0 && g1.D == d2t;
+  auto go = [&]<int KTc, int VECc, int Cc, int D2c, bool SAME1>() -> int {
     int grid = 0;
     if constexpr (D2c == -2) {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, true, -1, DenseMix>;
+      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, true, -1, -1, DenseMix>;
       if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
       kern<<<grid, Cc + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
     } else {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, GatherMix>;
+      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, (SAME1 ? D2c : -1), GatherMix>;
       if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
       kern<<<grid, Cc + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
     }
     *grid_out = grid;
     return check_launch(c, "outer_step_tma_kernel");
   };
+#define FGD_TMA_D(kt, v, cc, d)                                                             \
+  return same_d1 ? go.template operator()<kt, v, cc, d, true>() : go.template operator()<kt, v, cc, d, false>();
 #define FGD_TMA_CASE(kt, v, cc)                                                             \
   if (KT == kt && sh.vec == v && sh.consumers == cc) {                                      \
-    if (dense2) return go.template operator()<kt, v, cc, -2>();                             \
+    if (dense2) return go.template operator()<kt, v, cc, -2, false>();                      \
     switch (d2t) {                                                                          \
-      case 0: return go.template operator()<kt, v, cc, 0>();                                \
-      case 1: return go.template operator()<kt, v, cc, 1>();                                \
-      case 2: return go.template operator()<kt, v, cc, 2>();                                \
-      case 4: return go.template operator()<kt, v, cc, 4>();                                \
-      default: return go.template operator()<kt, v, cc, -1>();                              \
+      case 0: return go.template operator()<kt, v, cc, 0, false>();                         \
+      case 1: FGD_TMA_D(kt, v, cc, 1)                                                       \
+      case 2: FGD_TMA_D(kt, v, cc, 2)                                                       \
+      case 4: FGD_TMA_D(kt, v, cc, 4)                                                       \
+      default: return go.template operator()<kt, v, cc, -1, false>();                       \
     }                                                                                       \
   }
   FGD_TMA_CASE(0, 1, 128)
@@ -138,6 +143,7 @@ int launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix&
   FGD_TMA_CASE(32, 1, 256) FGD_TMA_CASE(32, 1, 128)
   FGD_TMA_CASE(64, 1, 128)
 #undef FGD_TMA_CASE
+#undef FGD_TMA_D
   return fail(c, FGD_ERR_UNSUPPORTED, "internal: no TMA kernel for this shape");
 }
 

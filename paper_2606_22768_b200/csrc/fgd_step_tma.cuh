@@ -77,7 +77,8 @@ constexpr int kMaxStages = 8;
 
 // D2T: compile-time neighbour count of a gather Mix2 (-1 = read at run time; ignored for a mean
 // or dense Mix2).
-template <int KT, int VEC, int CONSUMERS, bool DENSE2, int D2T, typename M2>
+// D1T: the same for a fused gather Mix1 (-1 = run time).
+template <int KT, int VEC, int CONSUMERS, bool DENSE2, int D2T, int D1T, typename M2>
 __global__ void __launch_bounds__(CONSUMERS + 32)
 outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
                       const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
@@ -286,7 +287,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
             if constexpr (XREGS) xm = xr[m];
             else xm = SCol<VEC>::ld(X, m * TPB + t);
           } else if (a.xsrc == XSRC_FUSED && m1.kind == KMIX_GATHER) {
-            xm = gather_row<VEC, TPB>(m1, m, A, t);
+            xm = gather_row<VEC, TPB, D1T>(m1, m, A, t);
           } else {
             xm = xv;
           }
