@@ -57,7 +57,7 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
     }                                                                                       \
   }
 #if FGD_TMA_GROUP == 0
-  FGD_TMA_CASE(0, 1, 128)
+  FGD_TMA_CASE(0, 2, 256) FGD_TMA_CASE(0, 1, 256) FGD_TMA_CASE(0, 1, 128)
   FGD_TMA_CASE(2, 4, 256) FGD_TMA_CASE(2, 4, 128)
   FGD_TMA_CASE(4, 4, 256) FGD_TMA_CASE(4, 4, 128)
 #elif FGD_TMA_GROUP == 1

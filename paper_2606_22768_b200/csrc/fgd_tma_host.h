@@ -48,7 +48,7 @@ struct TmaShape {
   int vec, consumers, stages;
 };
 const int kTmaShapes[][3] = {  // {KT, vec, consumers}, in order of preference per KT
-    {0, 1, 128},
+    {0, 2, 256}, {0, 1, 256}, {0, 1, 128},   // run-time K: widest tile whose two stages fit
     {2, 4, 256}, {2, 4, 128},
     {4, 4, 256}, {4, 4, 128},
     {8, 4, 256}, {8, 4, 128},
@@ -68,7 +68,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* ou
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
   const int K = c->K, KT = kt_of(K), NT = tma_n_tensors(a, KT, dense2);
-  const size_t budget = (size_t)c->max_smem_optin - 4096;  // static shared memory + slack
+  const size_t budget = (size_t)c->max_smem_optin - 6144;  // static shared memory (barriers, reduction buffer) + slack
   for (const auto& sh : kTmaShapes) {
     if (sh[0] != KT) continue;
     const int vec = sh[1], consumers = sh[2];
