@@ -108,6 +108,9 @@ __device__ __forceinline__ void tmem_ld_32(uint32_t taddr, float (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// XMAT: the Mix1 result is a [K, ld] matrix (a compile-time switch: its 32 extra registers per
+// thread would otherwise slow the common cases down).
+template <bool XMAT>
 __global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
@@ -213,6 +216,13 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       const bool live = col < P;
       float xv = 0.f;
       if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
+      float xr[XMAT ? H : 1];                      // a matrix-valued Mix1 result: this thread's rows, requested
+      if constexpr (XMAT) {                        // now so that they arrive behind the TMA wait and the MMA
+        if (live) {
+#pragma unroll
+          for (int m = 0; m < H; ++m) xr[m] = __ldcs(a.x + (size_t)(r0 + m) * ld + col);
+        }
+      }
       unsigned char* stage = base + (size_t)s * 3 * kTcBox;
       float* A = reinterpret_cast<float*>(stage);                 // theta_prev  -> g_lo operand
       float* B = reinterpret_cast<float*>(stage + kTcBox);        // theta_local -> g_hi operand
@@ -282,7 +292,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
 #pragma unroll
         for (int m = 0; m < H; ++m) v[m] = vs;
       }
-      if (a.xsrc != XSRC_VECTOR) xv = tsum * invK;
+      if (a.xsrc == XSRC_FUSED) xv = tsum * invK;
       if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
@@ -302,7 +312,9 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
 #pragma unroll
         for (int m = 0; m < H; ++m) {
           const float vn = fmaf(mu, v[m], gh[m]);
-          const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xv);
+          float xm = xv;
+          if constexpr (XMAT) xm = xr[m];
+          const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xm);
           __stcs(mom_col + (size_t)m * ld, vn);
           __stcs(new_col + (size_t)m * ld, tn);
           v[m] = tn;

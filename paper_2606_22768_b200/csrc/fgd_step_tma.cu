@@ -11,12 +11,12 @@ int fgd_launch_step_tma_g0(fgd_ctx*, const StepArgs&, bool, const GatherMix&, co
 int fgd_launch_step_tma_g1(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 int fgd_launch_step_tma_g2(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 
-// Tensor-core dense step: K = 64, Mix1 given as the averaged row or fused as a mean.
+// Tensor-core dense step: K = 64, Mix1 given (row or matrix) or fused as a mean.
 bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g1) {
   if (!dense2 || c->K != kTcK || !c->encode_tiled || a.n_ranges != 0) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
-  if (!(a.xsrc == XSRC_VECTOR || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
+  if (!(a.xsrc == XSRC_VECTOR || a.xsrc == XSRC_MATRIX || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
   return (size_t)c->max_smem_optin >= kTcSmem + 2048;
 }
 
@@ -33,9 +33,15 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   if (int rc = make_tensor_map(c, &tm, a.momentum, kTcCols)) return rc;
   const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
   int grid = 0;
-  auto kern = outer_step_dense_tc_kernel;
-  if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
-  kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  if (a.xsrc == XSRC_MATRIX) {
+    auto kern = outer_step_dense_tc_kernel<true>;
+    if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
+    kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  } else {
+    auto kern = outer_step_dense_tc_kernel<false>;
+    if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
+    kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  }
   *grid_out = grid;
   return check_launch(c, "outer_step_dense_tc_kernel");
 }
