@@ -66,6 +66,8 @@ def parse_args():
     ap.add_argument("--subset-frac", type=float, default=0.0,
                     help="variant: restrict Mix2 to about this fraction of the columns (three blocks)")
     ap.add_argument("--average-momentum", action="store_true", help="variant: GlobalM1S (needs Mix1 = mean)")
+    ap.add_argument("--chain-mix1", action="store_true",
+                    help="variant: the fused step also writes next round's global-average Mix1 (no Mix1 kernel)")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
@@ -264,16 +266,20 @@ def run_ours(args):
         cfg["name"] += f" [variant: Mix2 on {sum(b - a for a, b in ranges) / P:.0%} of the columns]"
     if args.average_momentum:
         cfg["name"] += " [variant: momentum averaged (GlobalM1S)]"
+    if args.chain_mix1:
+        cfg["name"] += " [variant: Mix1 (mean) of round r+1 emitted by the fused step of round r]"
 
     def one_round(r, ev_pair=None):
         m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
         m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
         drv.cd_sumsq = cd_log[r]
-        drv.launch_mix1(m1, theta)
+        if not (args.chain_mix1 and drv._pending is not None):
+            drv.launch_mix1(m1, theta)
         if ev_pair is not None:
             main.wait_event(drv._pending[0])     # keep the Mix1 wait out of the kernel's event pair
             ev_pair[0].record(main)
-        drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix2_ranges=ranges, average_momentum=args.average_momentum)
+        drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix2_ranges=ranges, average_momentum=args.average_momentum,
+                 emit_next_mix1=args.chain_mix1)
         if ev_pair is not None:
             ev_pair[1].record(main)
 

@@ -160,11 +160,19 @@ int fgd_outer_step(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* m
  *       optimizer state, v_m <- (1/K) sum_n v_n, before the Nesterov update.  Needs Mix1 to be
  *       the global average (x given as the averaged row, or mix1_fused of kind MEAN), else
  *       FGD_ERR_UNSUPPORTED.
+ *   x_next                  device [P] or NULL.  When Mix1 is the global average, next round's
+ *       Mix1 result x_{r+1} = (1/K) sum_m theta_new_m depends only on this step's output, and
+ *       the step already forms that column mean for the consensus term: with x_next the kernel
+ *       writes it out (4/K bytes per worker-parameter more), so the caller can skip the
+ *       separate fgd_mix of the next round.  Same value as launching Mix1 at the top of the
+ *       next round (Algorithm 1): nothing stale.  Must not overlap any other tensor, in
+ *       particular not the `x` this call reads.
  * opts == NULL is fgd_outer_step. */
 typedef struct {
   const int64_t* mix2_ranges;
   int32_t n_ranges;
   int32_t average_momentum;
+  float* x_next;
 } fgd_step_options;
 int fgd_outer_step_ex(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused,
                       const float* x, int x_is_vector, const float* theta_local,

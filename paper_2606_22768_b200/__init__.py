@@ -305,19 +305,23 @@ def fgd_outer_step(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x
 
 
 class _CStepOptions(ctypes.Structure):
-    _fields_ = [("mix2_ranges", ctypes.c_void_p), ("n_ranges", ctypes.c_int32), ("average_momentum", ctypes.c_int32)]
+    _fields_ = [("mix2_ranges", ctypes.c_void_p), ("n_ranges", ctypes.c_int32), ("average_momentum", ctypes.c_int32),
+                ("x_next", ctypes.c_void_p)]
 
 
 def fgd_outer_step_ex(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x, x_is_vector: bool,
                       theta_local, theta_prev, momentum, theta_new, lr: float = 0.7, mu: float = 0.9,
-                      cd_sumsq=None, mix2_ranges=None, average_momentum: bool = False, stream=None) -> None:
+                      cd_sumsq=None, mix2_ranges=None, average_momentum: bool = False, x_next=None,
+                      stream=None) -> None:
     """fgd_outer_step with the paper's two variants: Mix2 only inside the given (lo, hi) column
-    ranges (the "-subset" configurations) and/or the momentum averaged first (GlobalM1S)."""
+    ranges (the "-subset" configurations) and/or the momentum averaged first (GlobalM1S); with
+    ``x_next`` ([P]) the kernel also writes the column mean of theta_new, i.e. next round's
+    global-average Mix1 result."""
     ranges = None
     if mix2_ranges is not None:
         ranges = np.ascontiguousarray(np.asarray(mix2_ranges, dtype=np.int64).reshape(-1, 2))
     opts = _CStepOptions(None if ranges is None else ranges.ctypes.data, 0 if ranges is None else ranges.shape[0],
-                         int(bool(average_momentum)))
+                         int(bool(average_momentum)), _dev_ptr(x_next, "x_next", "torch.float32"))
     ctx._check(_lib.fgd_outer_step_ex(
         ctx._h, ctypes.byref(mix2.c()), None if mix1_fused is None else ctypes.byref(mix1_fused.c()),
         _dev_ptr(x, "x", "torch.float32"), int(bool(x_is_vector)),

@@ -217,6 +217,7 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   a.mu = (float)mu;
   a.n_ranges = 0;
   a.avg_momentum = 0;
+  a.x_next = nullptr;
   for (int i = 0; i < FGD_MAX_RANGES; ++i) a.range_lo[i] = a.range_hi[i] = 0;
   if (opts) {
     if (opts->n_ranges < 0 || opts->n_ranges > FGD_MAX_RANGES || (opts->n_ranges > 0 && !opts->mix2_ranges))
@@ -229,6 +230,13 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
       a.range_hi[i] = hi;
     }
     a.n_ranges = opts->n_ranges;
+    if (opts->x_next) {
+      const Range rn = vec_range(opts->x_next, c->P, sizeof(float));
+      if (overlap(rn, r_new) || overlap(rn, r_mom) || overlap(rn, r_prev) || overlap(rn, r_loc) ||
+          (x && overlap(rn, x_is_vector ? vec_range(x, c->P, sizeof(float)) : mat_range(x, K, c->P, c->ld))))
+        return fail(c, FGD_ERR_ALIAS, "fgd_outer_step_ex: x_next overlaps another tensor");
+      a.x_next = opts->x_next;
+    }
     if (opts->average_momentum) {
       const bool mean1 = mix1_fused ? mix1_fused->kind == FGD_MIX_MEAN : (x_is_vector != 0);
       if (!mean1) return fail(c, FGD_ERR_UNSUPPORTED, "fgd_outer_step_ex: average_momentum needs Mix1 to be the global average");
@@ -271,7 +279,7 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
     // (with one or two workers a tile is too little work per pipeline hand-off: AUTO keeps the register kernel)
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
-    const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x});
+    const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next});
     rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
       const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
       const size_t col = sizeof(float) * (size_t)K * kBlock * VECc;

@@ -51,6 +51,7 @@ struct StepArgs {
   // variants (fgd_outer_step_ex): Mix2 only inside column ranges; momentum averaged first
   int n_ranges;                          // 0 = Mix2 on every column
   int avg_momentum;                      // 1 = v_m <- mean_n v_n before the update
+  float* x_next;                         // [P] or nullptr: column mean of theta_new (next round's global-average Mix1)
   int64_t range_lo[FGD_MAX_RANGES];
   int64_t range_hi[FGD_MAX_RANGES];
 };

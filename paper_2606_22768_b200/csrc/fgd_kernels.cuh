@@ -415,6 +415,7 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
       }
     }
 
+    if (a.x_next) st_stream<VEC>(a.x_next + col, p_mul<VEC>(asum, invK));   // next round's global-average Mix1
     // ---- consensus distance of theta_new: squared deviation from the column mean
     if (want_cd) {
 #pragma unroll(KT > 0 ? KT : 4)

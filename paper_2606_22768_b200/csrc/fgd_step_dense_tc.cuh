@@ -321,11 +321,12 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           asum += tn;
         }
       }
-      if (want_cd) {                               // column mean over both halves, then squared deviations
+      if (want_cd || a.x_next) {                   // column mean over both halves, then squared deviations
         xchg[h][c] = asum;
         named_bar_sync(3, CONS);
         const float mean = (asum + xchg[h ^ 1][c]) * invK;
-        if (live) {
+        if (a.x_next && live && h == 0) __stcs(a.x_next + col, mean);   // next round's global-average Mix1
+        if (live && want_cd) {
 #pragma unroll
           for (int m = 0; m < H; ++m) {
             const float d = v[m] - mean;

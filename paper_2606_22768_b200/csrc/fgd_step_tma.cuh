@@ -324,6 +324,13 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
             finish_row(m, gh);
           }
         }
+        if (a.x_next) {                             // next round's global-average Mix1, for free
+          const Pack<VEC> xn = p_mul<VEC>(asum, invK);
+          if (whole) st_stream<VEC>(a.x_next + col, xn);
+          else
+            for (int q = 0; q < VEC; ++q)
+              if (col + q < P) a.x_next[col + q] = xn.v[q];
+        }
         // ---- phase 3: squared deviation of theta_new from its column mean
         if (want_cd) {
           const Pack<VEC> nmean = p_mul<VEC>(asum, -invK);

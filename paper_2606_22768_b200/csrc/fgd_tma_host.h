@@ -73,6 +73,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* ou
     if (sh[0] != KT) continue;
     const int vec = sh[1], consumers = sh[2];
     if (a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
+    if (a.x_next && (reinterpret_cast<uintptr_t>(a.x_next) % (sizeof(float) * vec)) != 0) continue;
     const size_t fixed = tma_fixed_smem(K, KT, dense2, consumers);
     const size_t stage = tma_stage_bytes(K, consumers * vec, NT);
     if (budget < fixed + 2 * stage) continue;

@@ -30,6 +30,7 @@ class OuterRound:
         self.side = torch.cuda.Stream(device=self.device)
         self.cd_sumsq = torch.zeros(K, dtype=torch.float64, device=self.device)
         self._x_vec = None
+        self._x_vec2 = None   # second [P] buffer: a step that emits next round's Mix1 writes the one it does not read
         self._x_mat = None
         self._pending = None  # (event, x tensor, x_is_vector)
 
@@ -54,15 +55,27 @@ class OuterRound:
     # ---- blocking part: wait for Mix1, then the fused outer step ---------------------------
     def step(self, mix2: MixDesc, theta_local, theta_prev, momentum, theta_new, lr: float = 0.7,
              mu: float = 0.9, mix1_fused: Optional[MixDesc] = None, want_cd: bool = True,
-             mix2_ranges=None, average_momentum: bool = False) -> None:
+             mix2_ranges=None, average_momentum: bool = False, emit_next_mix1: bool = False) -> None:
         """Fused outer step on the current stream.  Uses the pending side-stream Mix1 result,
         or computes Mix1 inside the kernel when ``mix1_fused`` is given.  ``mix2_ranges`` (column
         ranges Mix2 is restricted to) and ``average_momentum`` select the paper's "-subset" and
-        GlobalM1S variants."""
+        GlobalM1S variants.  With ``emit_next_mix1`` (Mix1 = global average) the step also writes
+        next round's Mix1 result -- the column mean of theta_new it forms anyway -- and leaves it
+        pending, so the next round needs no ``launch_mix1``."""
         cd = self.cd_sumsq if want_cd else None
+        x_next = None
+        if emit_next_mix1:
+            if self._x_vec is None:
+                self._x_vec = torch.empty(self.P, dtype=torch.float32, device=self.device)
+            if self._x_vec2 is None:
+                self._x_vec2 = torch.empty(self.P, dtype=torch.float32, device=self.device)
+            reading = self._pending[1] if self._pending is not None else None
+            x_next = self._x_vec2 if reading is self._x_vec else self._x_vec
         if mix1_fused is not None:
             fgd_outer_step_ex(self.ctx, mix2, mix1_fused, None, False, theta_local, theta_prev, momentum,
-                              theta_new, lr, mu, cd, mix2_ranges, average_momentum)
+                              theta_new, lr, mu, cd, mix2_ranges, average_momentum, x_next)
+            if x_next is not None:
+                self._pending = (torch.cuda.current_stream(self.device).record_event(), x_next, True)
             return
         if self._pending is None:
             raise RuntimeError("no Mix1 in flight: call launch_mix1() first or pass mix1_fused")
@@ -70,9 +83,12 @@ class OuterRound:
         self._pending = None
         torch.cuda.current_stream(self.device).wait_event(ev)
         fgd_outer_step_ex(self.ctx, mix2, None, x, is_vec, theta_local, theta_prev, momentum, theta_new,
-                          lr, mu, cd, mix2_ranges, average_momentum)
+                          lr, mu, cd, mix2_ranges, average_momentum, x_next)
         # the side stream may not overwrite x for the next round before this kernel has read it
-        self.side.wait_event(torch.cuda.current_stream(self.device).record_event())
+        done = torch.cuda.current_stream(self.device).record_event()
+        self.side.wait_event(done)
+        if x_next is not None:
+            self._pending = (done, x_next, True)
 
     def consensus(self, theta) -> torch.Tensor:
         fgd_consensus_distance(self.ctx, theta, self.cd_sumsq)

@@ -94,11 +94,12 @@ class Scenario:
 
     def __init__(self, K, P, mix1, mix2, *, ld=None, seed=0, sigmas=1e-3, worker_std=0.0, mode="factored",
                  in_place=True, lr=0.7, mu=0.9, v0_std=0.0, path=fgd.FGD_PATH_AUTO,
-                 mix2_ranges=None, average_momentum=False):
+                 mix2_ranges=None, average_momentum=False, chain_mix1=False):
         self.K, self.P, self.ld = K, P, P if ld is None else ld
         self.mix1, self.mix2, self.seed, self.mode, self.in_place = mix1, mix2, seed, mode, in_place
         self.lr, self.mu = lr, mu
         self.mix2_ranges, self.average_momentum = mix2_ranges, average_momentum
+        self.chain_mix1 = chain_mix1   # rounds > 0 take Mix1 (mean) from the previous step's x_next
         self.sigmas = np.broadcast_to(np.asarray(sigmas, dtype=np.float32), (K,)).copy()
         th0 = gen.theta0(seed, K, P, 0.02, worker_std)
         v0 = (gen.scaled_normal(seed, gen.TENSOR_MOMENTUM, 0, K, P, v0_std) if v0_std > 0
@@ -119,14 +120,15 @@ class Scenario:
             # stand-in for the inner steps: same fp32 drift bits on both sides
             drift = gen.scaled_normal(self.seed, gen.TENSOR_DRIFT, r, K, P, self.sigmas)
             fused = self.mode == "fused" or self.mix1[0] == "identity"
-            if not fused:
+            if not fused and not (self.chain_mix1 and r > 0):
                 self.drv.launch_mix1(m1_desc, self.full_prev)
             th_prev32 = self.g_prev.cpu().numpy()
             loc32 = th_prev32 + drift
             self.g_loc.copy_(torch.from_numpy(loc32))
             self.drv.step(m2_desc, self.full_loc, self.full_prev, self.full_v, self.full_new, self.lr, self.mu,
                           mix1_fused=m1_desc if fused else None, want_cd=True,
-                          mix2_ranges=self.mix2_ranges, average_momentum=self.average_momentum)
+                          mix2_ranges=self.mix2_ranges, average_momentum=self.average_momentum,
+                          emit_next_mix1=self.chain_mix1)
             torch.cuda.synchronize()
             # oracle, free running: its own float64 state plus the shared drift
             o_loc = self.o_theta + drift.astype(np.float64)

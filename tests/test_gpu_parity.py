@@ -300,6 +300,16 @@ def test_paper_variants(name, K, P, mix1, mix2, subset, avg, path, mode):
              mix2_ranges=_subset(P) if subset else None, average_momentum=avg).run(3)
 
 
+@pytest.mark.parametrize("K,P,mix2", [(16, 50001, ("ring",)), (8, 30000, ("xor",)), (64, 9000, ("dense", SINK64)),
+                                       (64, 5000, ("hypercube",)), (6, 7000, ("ring",)), (2, 4000, ("ring",))])
+@pytest.mark.parametrize("path", PATHS)
+def test_step_emits_next_rounds_global_average(K, P, mix2, path):
+    """Mix1 = global average chained through the fused step: round r writes x_{r+1} = mean(theta_new),
+    round r+1 reads it instead of running a Mix1 kernel.  Same values as Algorithm 1."""
+    ld = P + (4 - P % 4) % 4
+    Scenario(K, P, ("mean",), mix2, ld=ld, seed=8, path=path, chain_mix1=True, v0_std=1e-3).run(4)
+
+
 def test_variant_argument_errors():
     K, P = 4, 1024
     ctx = fgd.Context(K, P)
@@ -315,6 +325,10 @@ def test_variant_argument_errors():
     with pytest.raises(fgd.FgdError) as e:    # too many ranges
         fgd.fgd_outer_step_ex(ctx, ring, mean, None, False, b, a, c, d, mix2_ranges=[(4 * i, 4 * i + 4) for i in range(9)])
     assert e.value.status == fgd.FGD_ERR_INVALID_ARG
+    with pytest.raises(fgd.FgdError) as e:    # x_next may not be the x this call reads
+        xv = torch.zeros(P, device="cuda")
+        fgd.fgd_outer_step_ex(ctx, ring, None, xv, True, b, a, c, d, x_next=xv)
+    assert e.value.status == fgd.FGD_ERR_ALIAS
     with pytest.raises(fgd.FgdError) as e:    # momentum averaging belongs to a global Mix1
         fgd.fgd_outer_step_ex(ctx, ring, ring, None, False, b, a, c, d, average_momentum=True)
     assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
