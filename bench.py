@@ -34,7 +34,7 @@ METRIC = "outer_round_worker_params_per_s"
 UNIT = "worker-params/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# BASELINE.json configs (index = position in "configs", 1-based here)
+# the five benchmark configurations (1-based)
 CONFIGS = {
     1: dict(K=4, P=1 << 20, mix1=("mean",), mix2=("ring",), sig=(1e-3, 1e-3), p_fail=0.0,
             name="cfg1 K=4 P=2^20 Mix1=mean Mix2=ring"),
@@ -51,7 +51,7 @@ CONFIGS = {
 # DRAM bytes per worker-parameter of the fused outer-step kernel measured with ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch / (K*P) of that launch); the
 # capture it comes from is summarised under profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: 20.04}  # profiles/outer_step_tma_kernel_cfg3_16Mcols_ncu.md
+NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: 20.04, 5: 19.85}
 
 
 def parse_args():

@@ -9,7 +9,11 @@ one random matching whose pairs average (Sec. 3, "Gossip-based Mixing"; App. A,
 the table of (Mix1, Mix2) choices).  Its failure model is one sentence: a missed
 exchange gives weaker mixing instead of aborting the round (Sec. 1; Sec. 5.2).
 Everything else here (ring / hypercube / one-peer schedules, the Bernoulli edge
-mask, the two renormalisation rules, the hash) is this build's stated reading.
+mask, the two renormalisation rules, the hash) is this build's stated reading:
+``edge_mask`` and ``effective_weights`` are PARITY UNPINNED BY THE PAPER (it gives no
+formula for either); they are pinned only by what the mathematics fixes -- symmetry,
+double stochasticity, the drop rate, the all-alive / all-dead extremes, a hand-worked
+fixture -- and by bit-exact agreement with the library's independent implementation.
 
 Sparse form used throughout: ``nbr[m][j]`` = j-th neighbour of worker m or -1 for an
 empty slot, ``w[m][j]`` its base weight, ``w_self[m]`` the base self weight.
