@@ -1,4 +1,4 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+"""Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times.
 
 The [K, P] tensors are generated in HBM by the seeded generator's CUDA twin; because every value
 is a pure function of (seed, tensor, round, worker, column), the oracle regenerates any column
