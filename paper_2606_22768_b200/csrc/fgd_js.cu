@@ -55,6 +55,7 @@ js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t
     __syncthreads();
     const unsigned prefix = s_prefix;
     const unsigned hi_mask = pass == 3 ? 0u : (0xFFFFFFFFu << (8 * (pass + 1)));
+#pragma unroll 4
     for (int64_t i = tid; i < V; i += kSelBlock) {
       const uint32_t key = desc_key(row[i]);
       if ((key & hi_mask) == (prefix & hi_mask)) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1u);
@@ -87,6 +88,8 @@ js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t
     bool valid = i < V;
     if (valid) key = desc_key(row[i]);
     const bool is_eq = valid && key == target;
+    // almost every chunk of a large vocabulary holds no candidate at all: one barrier and move on
+    if (!__syncthreads_or(valid && key <= target)) continue;
     // block-wide exclusive scan of is_eq
     const unsigned eq_ballot = __ballot_sync(0xffffffffu, is_eq);
     if (lane == 0) warp_tot[0][warp] = __popc(eq_ballot);
