@@ -46,6 +46,26 @@ def make_mix(spec, K, rnd, seed, mix_id):
     if kind == "dense":
         W32 = np.asarray(spec[1], dtype=np.float32)
         return fgd.MixDesc.dense(W32), oracle.dense_W("dense", K, W=W32.astype(np.float64))
+    if kind == "circulant":   # neighbours m +- 1 .. m +- h (D = 2h slots), Metropolis weights 1/(1+2h)
+        h = spec[1]
+        p_fail = spec[2] if len(spec) > 2 else 0.0
+        renorm = spec[3] if len(spec) > 3 else fgd.FGD_RENORM_METROPOLIS
+        nbr = [[(m + s * d) % K for d in range(1, h + 1) for s in (-1, 1)] for m in range(K)]
+        w = [[1.0 / (1 + 2 * h)] * (2 * h) for _ in range(K)]
+        ws = [1.0 / (1 + 2 * h)] * K
+        d = fgd.MixDesc.sparse(nbr, w, ws)
+        w32 = np.array(w, dtype=np.float32).astype(np.float64).tolist()
+        ws32 = np.array(ws, dtype=np.float32).astype(np.float64).tolist()
+        mask = None
+        if p_fail > 0.0:
+            d = d.with_failures(seed, rnd, mix_id, p_fail, renorm)
+            mask = T.edge_mask(seed, rnd, mix_id, p_fail, nbr)
+            assert d.edge_mask.tolist() == mask
+        w_eff, ws_eff = T.effective_weights(nbr, w32, ws32, mask, renorm if mask is not None else T.RENORM_NONE)
+        return d, np.array(T.dense_from_sparse(nbr, w_eff, ws_eff), dtype=np.float64)
+    if kind == "isolated":    # a sparse descriptor with no neighbour slots at all (D = 0): W = I
+        d = fgd.MixDesc.sparse(np.zeros((K, 0), dtype=np.int32), np.zeros((K, 0), dtype=np.float32), np.ones(K, dtype=np.float32))
+        return d, oracle.dense_W("identity", K)
     if kind in ("ring", "xor", "hypercube", "matching"):
         p_fail = spec[1] if len(spec) > 1 else 0.0
         renorm = spec[2] if len(spec) > 2 else fgd.FGD_RENORM_METROPOLIS

@@ -128,6 +128,13 @@ STEP_CASES = [
     (3, 2000, ("matching",), ("mean",)),
     (2, 1000, ("mean",), ("ring",)),
     (1, 300, ("identity",), ("identity",)),
+    # degenerate / extreme descriptors
+    (16, 12000, ("mean",), ("circulant", 4)),                                   # FGD_MAX_D = 8 neighbour slots
+    (16, 9000, ("circulant", 4, 0.3), ("circulant", 4, 0.3)),                   # ... with failures, both mixes
+    (8, 5000, ("mean",), ("isolated",)),                                        # D = 0
+    (16, 7000, ("mean",), ("hypercube", 1.0)),                                  # every edge dropped: Mix2 = identity
+    (16, 7000, ("mean",), ("hypercube", 0.4, fgd.FGD_RENORM_NONE)),             # no renormalisation: rows sum to < 1
+    (16, 7000, ("ring", 0.5, fgd.FGD_RENORM_SELF_ABSORB), ("ring", 0.5, fgd.FGD_RENORM_SELF_ABSORB)),
 ]
 
 
@@ -380,6 +387,10 @@ def test_argument_errors():
     with pytest.raises(fgd.FgdError) as e:
         fgd.fgd_outer_step(ctx, ring, fgd.MixDesc.dense(np.eye(K)), None, False, b, a, c, d)
     assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+    with pytest.raises(fgd.FgdError):
+        fgd.Context(4, 0)            # empty tensors are rejected, not launched
+    with pytest.raises(fgd.FgdError):
+        fgd.Context(0, 10)
     with pytest.raises(fgd.FgdError):
         fgd.Context(65, 10)
     with pytest.raises(fgd.FgdError):
