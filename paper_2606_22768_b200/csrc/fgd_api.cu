@@ -260,9 +260,10 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   int rc = FGD_OK;
   FgdTmaShape shape{0, 0, 0};
   const bool can_tma = fgd_tma_eligible(c, a, dense2, &shape);
-  // K = 64: the tensor-core kernel is the fastest fused step we have at this worker count, and
-  // any mix is also a dense matrix -- so a gather / mean Mix2 is densified and takes it too.
-  bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, true, g1);
+  // Worker counts up to 64 without a compile-time fp32 kernel of their own: the tensor-core kernel
+  // is the fastest fused step we have there, and any mix is also a dense matrix -- so a gather /
+  // mean Mix2 is densified and takes it too.
+  bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, dense2, g1);
   if (can_tc && !dense2) {
     double Wd[FGD_MAX_K * FGD_MAX_K];
     if (fgd_dense_matrix(mix2, Wd) != FGD_OK) can_tc = false;
@@ -270,13 +271,15 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
       for (int m = 0; m < K; ++m)
         for (int n = 0; n < K; ++n) d2.Wt[n * K + m] = (float)Wd[m * K + n];
   }
-  if ((c->path == FGD_PATH_TMA || c->path == FGD_PATH_TMA_FP32) && !can_tma)
+  if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma))
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   if (can_tc && c->path != FGD_PATH_REGISTER) {
     rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
-  } else if (can_tma && c->path != FGD_PATH_REGISTER && !(c->path == FGD_PATH_AUTO && K <= 2)) {
-    // (with one or two workers a tile is too little work per pipeline hand-off: AUTO keeps the register kernel)
+  } else if (can_tma && c->path != FGD_PATH_REGISTER && !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && KT == 16)))) {
+    // (AUTO keeps the register kernel with one or two workers, where a tile is too little work per
+    // pipeline hand-off, and for a dense Mix2 at K = 16, where its all-register W g product measured
+    // 6.1 TB/s against 5.0 TB/s for the shared-memory version of the pipelined kernel)
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next});

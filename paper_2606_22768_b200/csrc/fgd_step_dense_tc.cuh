@@ -16,8 +16,8 @@
 // Nesterov update, the streaming stores and the consensus sums follow without any exchange.
 //
 // Pipeline per CTA (one per SM): a producer warp streams [K x 128] boxes of theta_prev,
-// theta_local and momentum into a 2-stage shared-memory ring with 2-D TMA loads; the four
-// consumer warps compute g = theta_prev - theta_local in registers, split it and write g_hi /
+// theta_local and momentum into a shared-memory ring (2 stages at K = 64, 4 at K = 32) with 2-D
+// TMA loads; the eight consumer warps (two threads per column, half of the workers each) compute g = theta_prev - theta_local in registers, split it and write g_hi /
 // g_lo IN PLACE over the theta_local / theta_prev boxes of the stage in the K-major core-matrix
 // operand layout (a thread's four consecutive workers are one 16-byte row of a core matrix, so
 // its stores are 128-bit and conflict-free); one thread issues the 3 x (K/8) MMAs and commits them to an
@@ -59,63 +59,60 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 lanes x 32 bit x 64 columns: thread i of the warp receives columns 0..63 of lane (base + i).
-__device__ __forceinline__ void tmem_ld_64(uint32_t taddr, float (&r)[64]) {
-  uint32_t* u = reinterpret_cast<uint32_t*>(r);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
-      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
-      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-        "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-        "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31]),
-        "=r"(u[32]), "=r"(u[33]), "=r"(u[34]), "=r"(u[35]), "=r"(u[36]), "=r"(u[37]), "=r"(u[38]), "=r"(u[39]),
-        "=r"(u[40]), "=r"(u[41]), "=r"(u[42]), "=r"(u[43]), "=r"(u[44]), "=r"(u[45]), "=r"(u[46]), "=r"(u[47]),
-        "=r"(u[48]), "=r"(u[49]), "=r"(u[50]), "=r"(u[51]), "=r"(u[52]), "=r"(u[53]), "=r"(u[54]), "=r"(u[55]),
-        "=r"(u[56]), "=r"(u[57]), "=r"(u[58]), "=r"(u[59]), "=r"(u[60]), "=r"(u[61]), "=r"(u[62]), "=r"(u[63])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-constexpr int kTcK = 64;            // workers (MMA K and N dimensions)
+constexpr int kTcMaxK = 64;         // most workers (MMA K and N dimensions)
+constexpr int kTcMinK = 17;         // fewest workers sent to this kernel (padding dominates below)
 constexpr int kTcCols = 128;        // columns per tile (MMA M dimension)
-constexpr int kTcHalf = kTcK / 2;   // workers per consumer thread: two threads share a column
-constexpr int kTcConsumers = 2 * kTcCols;
-constexpr int kTcStages = 2;
-constexpr int kTcTmemCols = 64;     // fp32 accumulator columns (= K), a power of two >= 32
-constexpr uint32_t kTcBox = kTcK * kTcCols * sizeof(float);   // 32 KB: one tensor of a stage
-constexpr uint32_t kTcWBytes = kTcK * kTcK * sizeof(float);   // 16 KB: one split of W
-// dynamic shared memory: alignment slack + stages + W_hi + W_lo
-constexpr size_t kTcSmem = 128 + (size_t)kTcStages * 3 * kTcBox + 2 * kTcWBytes;
+constexpr int kTcConsumers = 2 * kTcCols;   // two threads share a column, each owns half of the workers
+// Shapes.  KP = padded worker count (a multiple of 16: the MMA's N granularity at M = 128);
+// worker counts in between are zero-padded up to the next shape.
+template <int KP>
+struct TcShape {
+  static_assert(KP % 16 == 0 && KP >= 32 && KP <= kTcMaxK, "unsupported padded worker count");
+  static constexpr int kHalf = KP / 2;                                 // workers per consumer thread
+  static constexpr uint32_t kBox = KP * kTcCols * sizeof(float);       // one tensor of a stage
+  static constexpr uint32_t kWBytes = KP * KP * sizeof(float);         // one split of W
+  static constexpr uint32_t kSbo = KP * 32;                            // operand layout: bytes between 8-row groups
+  static constexpr int kTmemCols = KP <= 32 ? 32 : 64;                 // fp32 accumulator columns: a power of two >= 32
+  static constexpr int kStages = KP <= 32 ? 4 : 2;                     // what fits in 227 KB next to W_hi and W_lo
+  // dynamic shared memory: alignment slack + stages + W_hi + W_lo
+  static constexpr size_t kSmem = 128 + (size_t)kStages * 3 * kBox + 2 * kWBytes;
+};
+constexpr int tc_padded_k(int K) { return K <= 32 ? 32 : (K <= 48 ? 48 : 64); }
 
-// 32 lanes x 32 bit x 32 columns: thread i of the warp receives 32 consecutive columns of lane (base + i).
-__device__ __forceinline__ void tmem_ld_32(uint32_t taddr, float (&r)[32]) {
+// 32 lanes x 32 bit x 8 columns: thread i of the warp receives 8 consecutive columns of lane
+// (base + i).  No wait: tmem_ld_wait() makes the registers valid.
+__device__ __forceinline__ void tmem_ld_8(uint32_t taddr, float* r) {
   uint32_t* u = reinterpret_cast<uint32_t*>(r);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-        "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-        "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// N (a multiple of 8) consecutive accumulator columns of this thread's lane.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&r)[N]) {
+  static_assert(N % 8 == 0, "column count must be a multiple of 8");
+#pragma unroll
+  for (int j = 0; j < N; j += 8) tmem_ld_8(taddr + (uint32_t)j, &r[j]);
+  tmem_ld_wait();
 }
 
 // XMAT: the Mix1 result is a [K, ld] matrix (a compile-time switch: its 32 extra registers per
 // thread would otherwise slow the common cases down).
-template <bool XMAT>
+// FULL: exactly KP workers.  Otherwise the worker count KR < KP is a run-time value and the
+// problem is zero-padded to KP: the TMA boxes stay KP rows tall (rows at or beyond KR are outside
+// the tensor and arrive as zeros without touching HBM), W is padded with zero rows and columns,
+// and only the first KR rows are stored.
+template <int KP, bool XMAT, bool FULL>
 __global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                            const __grid_constant__ CUtensorMap tm_mom) {
-  constexpr int K = kTcK, T = kTcCols, H = kTcHalf, CONS = kTcConsumers, STAGES = kTcStages;
+  using Shape = TcShape<KP>;
+  constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
+  constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
+  const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];   // full[], empty[], mma
   __shared__ int abort_flag;
@@ -143,17 +140,17 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // B operand = W^T as an N x K (m x n) matrix, K-major, no swizzle: 8-row x 16-byte core
-  // matrices; core matrices adjacent in K are 128 B apart, adjacent in N 2048 B apart.
+  // matrices; core matrices adjacent in K are 128 B apart, adjacent in N SBO = 32 K bytes apart.
   for (int i = tid; i < K * K; i += CONS + 32) {
-    const int n = i / K, m = i % K;          // m2.Wt[n*K+m] = W[m][n]
-    const float w = m2.Wt[i];
+    const int n = i / K, m = i % K;          // m2.Wt[n*KR+m] = W[m][n]
+    const float w = (FULL || (n < KR && m < KR)) ? m2.Wt[n * KR + m] : 0.f;
     const float hi = to_tf32(w);
-    const uint32_t off = (uint32_t)(m >> 3) * 2048u + (uint32_t)(n >> 2) * 128u + (uint32_t)(m & 7) * 16u + (uint32_t)(n & 3) * 4u;
+    const uint32_t off = (uint32_t)(m >> 3) * SBO + (uint32_t)(n >> 2) * 128u + (uint32_t)(m & 7) * 16u + (uint32_t)(n & 3) * 4u;
     *reinterpret_cast<float*>(wb_hi + off) = hi;
     *reinterpret_cast<float*>(wb_lo + off) = w - hi;
   }
   if (warp == CONS / 32) {   // the producer warp owns tensor memory: allocate the accumulator columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTcTmemCols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)Shape::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // W operands are read by the MMA (async proxy)
@@ -196,16 +193,17 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   } else {
     // ===================================================== consumers
     // Two threads per column: thread (c, h) owns column c of the tile and the workers
-    // [32 h, 32 h + 32) -- eight consumer warps instead of four hide the shared-memory, TMEM and
-    // barrier latencies, and 32 instead of 64 values per array keep everything in registers.
+    // [H h, H h + H), H = K / 2 -- eight consumer warps instead of four hide the shared-memory,
+    // TMEM and barrier latencies, and half-length arrays keep everything in registers.
     const int c = tid & (T - 1), h = tid >> 7, r0 = h * H;
-    const float invK = 1.0f / (float)K;
+    const float invK = 1.0f / (float)KR;
+    const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
     const float lr = a.lr, mu = a.mu;
     const bool need_tsum = a.xsrc == XSRC_FUSED;                      // fused mean Mix1
     // A operand = g^T as an M x K (column x worker) matrix, K-major, no swizzle, same core-matrix
     // scheme as B: row c, four consecutive workers = one 16-byte core-matrix row, so a thread's
-    // 32 values go out as 8 conflict-free 128-bit stores.
-    const uint32_t op_row = (uint32_t)(c >> 3) * 2048u + (uint32_t)(c & 7) * 16u;
+    // H values go out as H / 4 conflict-free 128-bit stores.
+    const uint32_t op_row = (uint32_t)(c >> 3) * SBO + (uint32_t)(c & 7) * 16u;
     // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
     constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
     int64_t i = 0;
@@ -220,7 +218,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       if constexpr (XMAT) {                        // now so that they arrive behind the TMA wait and the MMA
         if (live) {
 #pragma unroll
-          for (int m = 0; m < H; ++m) xr[m] = __ldcs(a.x + (size_t)(r0 + m) * ld + col);
+          for (int m = 0; m < H; ++m)
+            if (FULL || m < hr) xr[m] = __ldcs(a.x + (size_t)(r0 + m) * ld + col);
         }
       }
       unsigned char* stage = base + (size_t)s * 3 * kTcBox;
@@ -273,8 +272,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           const uint32_t bb = prod == 2 ? b_lo : b_hi;
 #pragma unroll
           for (int ks = 0; ks < K / 8; ++ks) {
-            const uint64_t da = umma_desc(aa + (uint32_t)ks * 256u, 128u, 2048u, 0u);
-            const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, 2048u, 0u);
+            const uint64_t da = umma_desc(aa + (uint32_t)ks * 256u, 128u, SBO, 0u);
+            const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, SBO, 0u);
             umma_tf32(tmem_base, da, db, idesc, (prod | ks) ? 1u : 0u);
           }
         }
@@ -284,7 +283,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       float v[H];
 #pragma unroll
       for (int m = 0; m < H; ++m) v[m] = C[(r0 + m) * T + c];
-      if (a.avg_momentum) {                        // GlobalM1S option: v_m <- mean_n v_n (all 64 workers)
+      if (a.avg_momentum) {                        // GlobalM1S option: v_m <- mean_n v_n (all workers)
         float vs = 0.f;
 #pragma unroll
         for (int m = 0; m < H; ++m) vs += v[m] + C[((H - r0) + m) * T + c];
@@ -303,7 +302,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
-      tmem_ld_32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
+      tmem_ld_cols<H>(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
       // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
       float asum = 0.f;
       if (live) {
@@ -311,6 +310,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         float* const new_col = a.theta_new + (size_t)r0 * ld + col;
 #pragma unroll
         for (int m = 0; m < H; ++m) {
+          if (!FULL && m >= hr) break;
           const float vn = fmaf(mu, v[m], gh[m]);
           float xm = xv;
           if constexpr (XMAT) xm = xr[m];
@@ -329,6 +329,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         if (live && want_cd) {
 #pragma unroll
           for (int m = 0; m < H; ++m) {
+            if (!FULL && m >= hr) break;
             const float d = v[m] - mean;
             sacc[m] = fmaf(d, d, sacc[m]);
           }
@@ -342,7 +343,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   __syncthreads();
   if (warp == CONS / 32) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTcTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Shape::kTmemCols) : "memory");
   }
   if (want_cd) {
     double* red = reinterpret_cast<double*>(base);    // [CONS/32][H]: warps 0-3 hold workers 0-31, warps 4-7 workers 32-63
@@ -356,12 +357,12 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       }
     }
     __syncthreads();
-    if (tid < K) {
+    if (tid < KR) {
       const int hh = tid / H, mm = tid % H;
       double d = 0.0;
 #pragma unroll
       for (int w = 0; w < T / 32; ++w) d += red[(hh * (T / 32) + w) * H + mm];
-      a.partials[(size_t)blockIdx.x * K + tid] = d;
+      a.partials[(size_t)blockIdx.x * KR + tid] = d;
     }
   }
 }

@@ -11,13 +11,37 @@ int fgd_launch_step_tma_g0(fgd_ctx*, const StepArgs&, bool, const GatherMix&, co
 int fgd_launch_step_tma_g1(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 int fgd_launch_step_tma_g2(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 
-// Tensor-core dense step: K = 64, Mix1 given (row or matrix) or fused as a mean.
-bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g1) {
-  if (!dense2 || c->K != kTcK || !c->encode_tiled || a.n_ranges != 0) return false;
+// Tensor-core dense step: Mix1 given (row or matrix) or fused as a mean; K = 64 and every worker
+// count in [17, 63] that has no compile-time fp32 kernel of its own (zero-padded to 32, 48 or 64),
+// plus K = 32 when Mix2 really is dense (`really_dense`: the caller's matrix, not a densified gather).
+bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, const GatherMix& g1) {
+  const int K = c->K;
+  if (K > kTcMaxK || K < kTcMinK) return false;
+  if (kt_of(K) == 16 || (kt_of(K) == 32 && !really_dense)) return false;
+  if (!c->encode_tiled || a.n_ranges != 0) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (!(a.xsrc == XSRC_VECTOR || a.xsrc == XSRC_MATRIX || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
-  return (size_t)c->max_smem_optin >= kTcSmem + 2048;
+  return (size_t)c->max_smem_optin >= TcShape<kTcMaxK>::kSmem + 2048;
+}
+
+template <int KP>
+static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, const GatherMix& g1, cudaStream_t st, int* grid) {
+  using Shape = TcShape<KP>;
+  const StepArgs& a = ta.s;
+  CUtensorMap tp, tl, tm;
+  if (int rc = make_tensor_map(c, &tp, a.theta_prev, kTcCols, KP)) return rc;
+  if (int rc = make_tensor_map(c, &tl, a.theta_local, kTcCols, KP)) return rc;
+  if (int rc = make_tensor_map(c, &tm, a.momentum, kTcCols, KP)) return rc;
+  const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
+  auto launch = [&](auto kern) -> int {
+    if (int r = persistent_grid(c, kern, kTcConsumers + 32, Shape::kSmem, ntiles, grid)) return r;
+    kern<<<*grid, kTcConsumers + 32, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm);
+    return FGD_OK;
+  };
+  const bool xmat = a.xsrc == XSRC_MATRIX, full = c->K == KP;
+  return xmat ? (full ? launch(outer_step_dense_tc_kernel<KP, true, true>) : launch(outer_step_dense_tc_kernel<KP, true, false>))
+              : (full ? launch(outer_step_dense_tc_kernel<KP, false, true>) : launch(outer_step_dense_tc_kernel<KP, false, false>));
 }
 
 int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, const GatherMix& g1, cudaStream_t st,
@@ -26,23 +50,13 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   ta.s = a;
   ta.status = c->status;
   ta.n_tensors = 3;
-  ta.stages = kTcStages;
-  CUtensorMap tp, tl, tm;
-  if (int rc = make_tensor_map(c, &tp, a.theta_prev, kTcCols)) return rc;
-  if (int rc = make_tensor_map(c, &tl, a.theta_local, kTcCols)) return rc;
-  if (int rc = make_tensor_map(c, &tm, a.momentum, kTcCols)) return rc;
-  const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
-  int grid = 0;
-  if (a.xsrc == XSRC_MATRIX) {
-    auto kern = outer_step_dense_tc_kernel<true>;
-    if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
-    kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
-  } else {
-    auto kern = outer_step_dense_tc_kernel<false>;
-    if (int r = persistent_grid(c, kern, kTcConsumers + 32, kTcSmem, ntiles, &grid)) return r;
-    kern<<<grid, kTcConsumers + 32, kTcSmem, st>>>(ta, d2, g1, tp, tl, tm);
+  int rc = FGD_OK;
+  switch (tc_padded_k(c->K)) {
+    case 32: ta.stages = TcShape<32>::kStages; rc = launch_tc<32>(c, ta, d2, g1, st, grid_out); break;
+    case 48: ta.stages = TcShape<48>::kStages; rc = launch_tc<48>(c, ta, d2, g1, st, grid_out); break;
+    default: ta.stages = TcShape<64>::kStages; rc = launch_tc<64>(c, ta, d2, g1, st, grid_out); break;
   }
-  *grid_out = grid;
+  if (rc) return rc;
   return check_launch(c, "outer_step_dense_tc_kernel");
 }
 

@@ -15,8 +15,8 @@ bool fgd_tma_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, Fgd
 int fgd_launch_step_tma(fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g2,
                         const fgd::DenseMix& d2, const fgd::GatherMix& g1, FgdTmaShape shape, cudaStream_t st,
                         int* grid_out);
-// Dense Mix2 on the tensor cores (K = 64).
-bool fgd_tc_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g1);
+// Dense Mix2 on the tensor cores (17 <= K <= 64, padded to 32 / 48 / 64 workers).
+bool fgd_tc_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool really_dense, const fgd::GatherMix& g1);
 int fgd_launch_step_dense_tc(fgd_ctx* c, const fgd::StepArgs& a, const fgd::DenseMix& d2, const fgd::GatherMix& g1,
                              cudaStream_t st, int* grid_out);
 #endif

@@ -17,11 +17,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 // 2-D map of a [K, ld] fp32 matrix restricted to its first P columns; box = boxc columns x K rows.
-// Columns at or beyond P read as zero.
-int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc) {
+// Columns at or beyond P read as zero.  box_rows > K asks for a taller box: its rows at or beyond K
+// lie outside the tensor and are filled with zeros too.
+int make_tensor_map(fgd_ctx* c, CUtensorMap* map, const float* base, int boxc, int box_rows = 0) {
   const cuuint64_t dims[2] = {(cuuint64_t)c->P, (cuuint64_t)c->K};
   const cuuint64_t strides[1] = {(cuuint64_t)c->ld * sizeof(float)};
-  const cuuint32_t box[2] = {(cuuint32_t)boxc, (cuuint32_t)c->K};
+  const cuuint32_t box[2] = {(cuuint32_t)boxc, (cuuint32_t)(box_rows > 0 ? box_rows : c->K)};
   const cuuint32_t estr[2] = {1, 1};
   CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(
       map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,

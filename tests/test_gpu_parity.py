@@ -135,6 +135,14 @@ STEP_CASES = [
     (16, 7000, ("mean",), ("hypercube", 1.0)),                                  # every edge dropped: Mix2 = identity
     (16, 7000, ("mean",), ("hypercube", 0.4, fgd.FGD_RENORM_NONE)),             # no renormalisation: rows sum to < 1
     (16, 7000, ("ring", 0.5, fgd.FGD_RENORM_SELF_ABSORB), ("ring", 0.5, fgd.FGD_RENORM_SELF_ABSORB)),
+    # worker counts between the compile-time kernels: zero-padded onto the 64-worker tensor-core kernel
+    (48, 9001, ("mean",), ("dense", gen.sinkhorn_W(3, 48))),
+    (48, 5000, ("ring",), ("ring", 0.2)),
+    (63, 4100, ("mean",), ("dense", gen.sinkhorn_W(4, 63))),
+    (33, 4099, ("ring",), ("matching",)),
+    (24, 7000, ("mean",), ("dense", gen.sinkhorn_W(5, 24))),
+    (17, 6002, ("matching",), ("ring",)),
+    (40, 3000, ("mean",), ("mean",)),
 ]
 
 
@@ -157,6 +165,12 @@ def test_outer_step_single_call(K, P, mix1, mix2, mode, path):
     cd = torch.zeros(K, dtype=torch.float64, device="cuda")
     ctx = fgd.Context(K, P, ld)
     fgd.fgd_set_path(ctx, path)
+    if K == 63 and path == fgd.FGD_PATH_TMA_FP32:
+        # two pipeline stages of 63 workers do not fit in shared memory: a forced path says so
+        with pytest.raises(fgd.FgdError) as e:
+            fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+        assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+        return
     if mode == "x_given":
         vec = mix1[0] == "mean"
         x = torch.empty(P if vec else (K, ld), dtype=torch.float32, device="cuda")
@@ -295,6 +309,8 @@ VARIANTS = [
     ("dense-subset", 64, 6000, ("mean",), ("dense", SINK64), True, False),
     ("dense-GlobalM1S", 64, 5000, ("mean",), ("dense", SINK64), False, True),
     ("dense16-subset", 16, 8000, ("ring",), ("dense", gen.sinkhorn_W(1, 16)), True, False),
+    ("dense48-GlobalM1S", 48, 5000, ("mean",), ("dense", gen.sinkhorn_W(3, 48)), False, True),
+    ("ring40-GlobalM1S", 40, 4001, ("mean",), ("ring",), False, True),
 ]
 
 
@@ -308,7 +324,8 @@ def test_paper_variants(name, K, P, mix1, mix2, subset, avg, path, mode):
 
 
 @pytest.mark.parametrize("K,P,mix2", [(16, 50001, ("ring",)), (8, 30000, ("xor",)), (64, 9000, ("dense", SINK64)),
-                                       (64, 5000, ("hypercube",)), (6, 7000, ("ring",)), (2, 4000, ("ring",))])
+                                       (64, 5000, ("hypercube",)), (6, 7000, ("ring",)), (2, 4000, ("ring",)),
+                                       (48, 6001, ("ring",)), (20, 5000, ("dense", gen.sinkhorn_W(6, 20)))])
 @pytest.mark.parametrize("path", PATHS)
 def test_step_emits_next_rounds_global_average(K, P, mix2, path):
     """Mix1 = global average chained through the fused step: round r writes x_{r+1} = mean(theta_new),
