@@ -98,18 +98,40 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&r)[N]) {
   tmem_ld_wait();
 }
 
-// XMAT: the Mix1 result is a [K, ld] matrix (a compile-time switch: its 32 extra registers per
-// thread would otherwise slow the common cases down).
+// Sparse Mix1 of the rows [r0, r0 + H) of one column from a staged [K][T] box of theta_prev.
+// DJ >= the used slot count: unused slots point at the row itself with weight 0, padded rows have
+// all-zero weights, so neither needs a branch; all loads of a row are issued before its FMAs.
+template <int DJ, int H, int T>
+__device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A, int r0, int c, float (&xr)[H]) {
+#pragma unroll
+  for (int m = 0; m < H; ++m) {
+    const int r = r0 + m;
+    float t[DJ > 0 ? DJ : 1];
+#pragma unroll
+    for (int j = 0; j < DJ; ++j) t[j] = A[m1.nbr[r * FGD_MAX_D + j] * T + c];
+    float acc = m1.w_self[r] * A[r * T + c];
+#pragma unroll
+    for (int j = 0; j < DJ; ++j) acc = fmaf(m1.w[r * FGD_MAX_D + j], t[j], acc);
+    xr[m] = acc;
+  }
+}
+
+// XM: where the Mix1 result x comes from.  0 = one value per column (a given row, or the column
+// mean of theta_prev computed here); 1 = a given [K, ld] matrix; 2 = a sparse (gossip) Mix1 fused
+// into this kernel: x_m = w_self[m] theta_prev[m] + sum_j w[m][j] theta_prev[nbr[m][j]], gathered
+// from the theta_prev box of the stage before the operands overwrite it.  (A compile-time switch:
+// the per-row x costs up to 32 extra registers per thread, which would slow the common case down.)
 // FULL: exactly KP workers.  Otherwise the worker count KR < KP is a run-time value and the
 // problem is zero-padded to KP: the TMA boxes stay KP rows tall (rows at or beyond KR are outside
 // the tensor and arrive as zeros without touching HBM), W is padded with zero rows and columns,
 // and only the first KR rows are stored.
-template <int KP, bool XMAT, bool FULL>
+template <int KP, int XM, bool FULL>
 __global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                            const __grid_constant__ CUtensorMap tm_mom) {
   using Shape = TcShape<KP>;
+  constexpr bool XMAT = XM != 0;                    // x differs from row to row
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
   constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
   const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
@@ -199,7 +221,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     const float invK = 1.0f / (float)KR;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
     const float lr = a.lr, mu = a.mu;
-    const bool need_tsum = a.xsrc == XSRC_FUSED;                      // fused mean Mix1
+    const bool need_tsum = XM == 0 && a.xsrc == XSRC_FUSED;           // fused mean Mix1
     // A operand = g^T as an M x K (column x worker) matrix, K-major, no swizzle, same core-matrix
     // scheme as B: row c, four consecutive workers = one 16-byte core-matrix row, so a thread's
     // H values go out as H / 4 conflict-free 128-bit stores.
@@ -215,7 +237,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       float xv = 0.f;
       if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
       float xr[XMAT ? H : 1];                      // a matrix-valued Mix1 result: this thread's rows, requested
-      if constexpr (XMAT) {                        // now so that they arrive behind the TMA wait and the MMA
+      if constexpr (XM == 1) {                     // now so that they arrive behind the TMA wait and the MMA
         if (live) {
 #pragma unroll
           for (int m = 0; m < H; ++m)
@@ -240,6 +262,14 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         if (need_tsum) {                           // the column mean needs the other half too
 #pragma unroll
           for (int n = 0; n < H; ++n) tsum += A[((H - r0) + n) * T + c];
+        }
+        if constexpr (XM == 2) {                   // gossip Mix1 of this thread's rows, from the stage
+          const int D1 = m1.D;                     // (uniform) -> a fully unrolled gather per slot count
+          if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, xr);
+          else if (D1 == 1) tc_gather_x<1, H, T>(m1, A, r0, c, xr);
+          else if (D1 == 2) tc_gather_x<2, H, T>(m1, A, r0, c, xr);
+          else if (D1 <= 4) tc_gather_x<4, H, T>(m1, A, r0, c, xr);
+          else tc_gather_x<FGD_MAX_D, H, T>(m1, A, r0, c, xr);
         }
       } else {
         *(volatile int*)&abort_flag = 1;
@@ -291,7 +321,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
 #pragma unroll
         for (int m = 0; m < H; ++m) v[m] = vs;
       }
-      if (a.xsrc == XSRC_FUSED) xv = tsum * invK;
+      if (need_tsum) xv = tsum * invK;
       if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);

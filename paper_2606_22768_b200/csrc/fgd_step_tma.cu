@@ -11,7 +11,7 @@ int fgd_launch_step_tma_g0(fgd_ctx*, const StepArgs&, bool, const GatherMix&, co
 int fgd_launch_step_tma_g1(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 int fgd_launch_step_tma_g2(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 
-// Tensor-core dense step: Mix1 given (row or matrix) or fused as a mean; K = 64 and every worker
+// Tensor-core dense step: Mix1 given (row or matrix) or fused (mean or gossip); K = 64 and every worker
 // count in [17, 63] that has no compile-time fp32 kernel of its own (zero-padded to 32, 48 or 64),
 // plus K = 32 when Mix2 really is dense (`really_dense`: the caller's matrix, not a densified gather).
 bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, const GatherMix& g1) {
@@ -21,7 +21,6 @@ bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, con
   if (!c->encode_tiled || a.n_ranges != 0) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
-  if (!(a.xsrc == XSRC_VECTOR || a.xsrc == XSRC_MATRIX || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
   return (size_t)c->max_smem_optin >= TcShape<kTcMaxK>::kSmem + 2048;
 }
 
@@ -39,9 +38,13 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
     kern<<<*grid, kTcConsumers + 32, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm);
     return FGD_OK;
   };
-  const bool xmat = a.xsrc == XSRC_MATRIX, full = c->K == KP;
-  return xmat ? (full ? launch(outer_step_dense_tc_kernel<KP, true, true>) : launch(outer_step_dense_tc_kernel<KP, true, false>))
-              : (full ? launch(outer_step_dense_tc_kernel<KP, false, true>) : launch(outer_step_dense_tc_kernel<KP, false, false>));
+  const bool full = c->K == KP;
+  const int xm = a.xsrc == XSRC_MATRIX ? 1 : ((a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER) ? 2 : 0);
+  switch (xm) {
+    case 1: return full ? launch(outer_step_dense_tc_kernel<KP, 1, true>) : launch(outer_step_dense_tc_kernel<KP, 1, false>);
+    case 2: return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
+    default: return full ? launch(outer_step_dense_tc_kernel<KP, 0, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false>);
+  }
 }
 
 int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, const GatherMix& g1, cudaStream_t st,

