@@ -129,7 +129,7 @@ template <int KP, int XM, bool FULL>
 __global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
-                           const __grid_constant__ CUtensorMap tm_mom) {
+                           const __grid_constant__ CUtensorMap tm_mom, const __grid_constant__ CUtensorMap tm_x) {
   using Shape = TcShape<KP>;
   constexpr bool XMAT = XM != 0;                    // x differs from row to row
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
@@ -204,6 +204,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         tma_load_2d(dst, &tm_prev, c0, 0, full, policy);
         tma_load_2d(dst + kTcBox, &tm_local, c0, 0, full, policy);
         tma_load_2d(dst + 2 * kTcBox, &tm_mom, c0, 0, full, policy);
+        // a matrix-valued x is read by the consumers straight into registers: have its box waiting in L2
+        if (XM == 1 && ta.n_tensors == 4) tma_prefetch_2d(&tm_x, c0, 0);
       }
       if (!ok) {
         *(volatile int*)&abort_flag = 1;

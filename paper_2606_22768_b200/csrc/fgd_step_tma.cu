@@ -28,14 +28,17 @@ template <int KP>
 static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, const GatherMix& g1, cudaStream_t st, int* grid) {
   using Shape = TcShape<KP>;
   const StepArgs& a = ta.s;
-  CUtensorMap tp, tl, tm;
+  CUtensorMap tp, tl, tm, tx;
   if (int rc = make_tensor_map(c, &tp, a.theta_prev, kTcCols, KP)) return rc;
   if (int rc = make_tensor_map(c, &tl, a.theta_local, kTcCols, KP)) return rc;
   if (int rc = make_tensor_map(c, &tm, a.momentum, kTcCols, KP)) return rc;
+  tx = tp;                                    // n_tensors == 4: x has a map of its own (L2 prefetch only)
+  if (ta.n_tensors == 4)
+    if (int rc = make_tensor_map(c, &tx, a.x, kTcCols, KP)) return rc;
   const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
   auto launch = [&](auto kern) -> int {
     if (int r = persistent_grid(c, kern, kTcConsumers + 32, Shape::kSmem, ntiles, grid)) return r;
-    kern<<<*grid, kTcConsumers + 32, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm);
+    kern<<<*grid, kTcConsumers + 32, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm, tx);
     return FGD_OK;
   };
   const bool full = c->K == KP;
@@ -52,7 +55,7 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   TmaStepArgs ta;
   ta.s = a;
   ta.status = c->status;
-  ta.n_tensors = 3;
+  ta.n_tensors = (a.xsrc == XSRC_MATRIX && aligned16(a.x)) ? 4 : 3;
   int rc = FGD_OK;
   switch (tc_padded_k(c->K)) {
     case 32: ta.stages = TcShape<32>::kStages; rc = launch_tc<32>(c, ta, d2, g1, st, grid_out); break;
