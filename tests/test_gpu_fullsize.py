@@ -100,3 +100,45 @@ def test_full_size_config(cfg_id, rounds):
     assert_cd_close(out, ref, WIDTH, "window consensus")
     del theta, local, mom
     torch.cuda.empty_cache()
+
+
+def test_more_than_2_to_31_columns():
+    """Maximum sizes: P just above 2^31 columns (64-bit column arithmetic end to end; the TMA kernels'
+    32-bit box coordinates do not reach that far, so AUTO must pick the register kernels and a forced
+    TMA path must refuse).  K = 3 ring, 2 rounds, sampled blocks around 0, 2^31 and the ragged end."""
+    K, P, seed = 3, (1 << 31) + 4102, 11
+    need = 3 * K * P * 4 + P * 4 + (2 << 30)
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip("not enough free HBM for this size")
+    sig = np.full(K, 1e-3, np.float32)
+    theta = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    local = torch.empty_like(theta)
+    mom = torch.zeros_like(theta)
+    inputs_gpu.theta0(theta, seed)
+    drv = OuterRound(K, P)
+    blocks = [0, (1 << 31) - 700, (1 << 31) + 2000, P - WIDTH, (1 << 30) + 12345]
+    o_theta = {p0: gen.theta0(seed, K, P, p0=p0, p1=p0 + WIDTH).astype(np.float64) for p0 in blocks}
+    o_v = {p0: np.zeros((K, WIDTH)) for p0 in blocks}
+    cd_alone = torch.zeros(K, dtype=torch.float64, device="cuda")
+    for r in range(2):
+        d1, W1 = make_mix(("mean",), K, r, seed, 1)
+        d2, W2 = make_mix(("ring", 0.2), K, r, seed, 2)
+        drv.launch_mix1(d1, theta)
+        inputs_gpu.local_steps(local, theta, sig, seed, r)
+        drv.step(d2, local, theta, mom, theta, 0.7, 0.9)
+        fgd.fgd_consensus_distance(drv.ctx, theta, cd_alone)
+        torch.cuda.synchronize()
+        fused, alone = drv.cd_sumsq.cpu().numpy(), cd_alone.cpu().numpy()
+        assert np.all(np.abs(fused - alone) <= 2e-6 * np.abs(alone)), f"round {r}: fused {fused} vs stand-alone {alone}"
+        for p0 in blocks:
+            drift = gen.scaled_normal(seed, gen.TENSOR_DRIFT, r, K, P, sig, p0, p0 + WIDTH).astype(np.float64)
+            o_theta[p0], o_v[p0] = oracle.outer_round(W1, W2, o_theta[p0], o_theta[p0] + drift, o_v[p0], 0.7, 0.9)
+            assert_param_close(theta[:, p0:p0 + WIDTH], o_theta[p0], f"round {r} theta_new block {p0}")
+            assert_param_close(mom[:, p0:p0 + WIDTH], o_v[p0], f"round {r} momentum block {p0}")
+    fgd.fgd_device_status(drv.ctx)
+    fgd.fgd_set_path(drv.ctx, fgd.FGD_PATH_TMA)
+    with pytest.raises(fgd.FgdError) as e:
+        fgd.fgd_outer_step(drv.ctx, d2, d1, None, False, local, theta, mom, theta, 0.7, 0.9, None)
+    assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
+    del theta, local, mom
+    torch.cuda.empty_cache()
