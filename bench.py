@@ -146,13 +146,16 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------- CPU oracle leg
-def oracle_leg(cfg, steps, warmup, seed=0, sample_cols=1 << 23):
+def oracle_leg(cfg, steps, warmup, seed=0, sample_cols=1 << 23, threads=0):
     """Times the float64 oracle, as it stands, on a bounded column sample of the workload."""
     import oracle
     from fgd_inputs import gen
     from oracle import topology as T
     K = cfg["K"]
     Ps = min(cfg["P"], sample_cols)
+    all_threads = oracle.num_threads()
+    if threads > 0:
+        oracle.set_num_threads(threads)
     sig = gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1] else np.full(K, cfg["sig"][0], np.float32)
     theta = gen.theta0(seed, K, Ps).astype(np.float64)
     v = np.zeros((K, Ps))
@@ -181,7 +184,9 @@ def oracle_leg(cfg, steps, warmup, seed=0, sample_cols=1 << 23):
         if r >= warmup:
             times.append(time.perf_counter() - t0)
     sec = sum(times) / len(times)
-    return {"value": K * Ps / sec, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    used = oracle.num_threads()
+    oracle.set_num_threads(all_threads)
+    return {"value": K * Ps / sec, "unit": UNIT, "cores": used, "kind": "oracle",
             "sample": f"first {Ps} of {cfg['P']} columns, all K={K} workers, {len(times)} round(s), "
                       f"{sec:.3f} s per round (round arithmetic + consensus sums only)"}, sec
 
@@ -323,8 +328,9 @@ def run_ours(args):
     tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if tr is None else tr * K * P,
-                "kernel": "outer_step_dense_tc_kernel" if (cfg["mix2"][0] == "dense" and K == 64) else "outer_step_tma_kernel",
-                "kernel_ms": kern_ms, "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
+                "kernel": "outer_step_dense_tc_kernel" if K == 64 else "outer_step_tma_kernel",
+                "kernel_ms": kern_ms, "kernel_ms_median": statistics.median(kern_times),
+                "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
                 "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / 8000.0}
 
@@ -345,6 +351,8 @@ def run_ours(args):
     if rank == 0:
         # context: the same STREAM-style copy the pool's peak was measured with, on THIS box, now
         roofline["copy_gbs_this_box"] = copy_bandwidth(torch, dev)
+    if rank == 0 and 3 * K * P * 4 <= 4 * 126e6:
+        line["latency"] = latency_leg(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, dev)
     if rank == 0 and not args.no_overlap:
         line["overlap"] = overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, dense_W)
     if not args.no_e2e:
@@ -352,6 +360,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         del theta, local, mom
         line["cpu_baseline"] = oracle_leg(cfg, 4, 1)[0]
+        line["cpu_baseline"]["value_1thread"] = oracle_leg(cfg, 1, 0, sample_cols=1 << 19, threads=1)[0]["value"]
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -484,6 +493,33 @@ def overlap_model(torch, fgd, inputs_gpu, drv, cfg, theta, local, sig, seed, den
     out = {"mix1_alone_ms": timed(mix1_only), "standin_compute_alone_ms": timed(standin_only),
            "overlapped_ms": timed(both)}
     drv._pending = None
+    return out
+
+
+def latency_leg(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, dev, reps=1000):
+    """L2-resident configuration: the fused outer step is launch- and latency-bound, not an HBM
+    number.  Times `reps` single launches (x given, consensus sums on) back to back with the working
+    set hot in L2, and again with a 512 MB write between launches that evicts it."""
+    K, P = cfg["K"], cfg["P"]
+    main = torch.cuda.current_stream(dev)
+    m2 = mix_desc(fgd, cfg["mix2"], cfg, 0, seed, 2, dense_W)
+    x = torch.zeros(P, dtype=torch.float32, device=dev)
+    cd = torch.zeros(K, dtype=torch.float64, device=dev)
+    flush = torch.empty(128 << 20, dtype=torch.float32, device=dev)
+    out = {"reps": reps, "unit": "us", "call": "fgd_outer_step, x given as [P], with consensus sums"}
+    for name, do_flush in (("l2_hot", False), ("l2_flushed", True)):
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i in range(-10, reps):
+            if do_flush:
+                flush.zero_()
+            if i >= 0:
+                pairs[i][0].record(main)
+            fgd.fgd_outer_step(drv.ctx, m2, None, x, True, local, theta, mom, theta, 0.7, 0.9, cd)
+            if i >= 0:
+                pairs[i][1].record(main)
+        torch.cuda.synchronize()
+        us = sorted(a.elapsed_time(b) * 1e3 for a, b in pairs)
+        out[name] = {"median": us[len(us) // 2], "best": us[0], "p95": us[int(0.95 * len(us))]}
     return out
 
 
