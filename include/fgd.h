@@ -37,6 +37,11 @@
  *  - fgd_outer_step (with cd_sumsq) and fgd_consensus_distance use the context's small
  *    partial-sum scratch: two such calls on one context must be ordered on the GPU
  *    (same stream or an event); all other calls may overlap freely.
+ *  - Stream capture: after one eager call with the same context, mix kind and argument
+ *    shapes (it sizes the launch), fgd_outer_grad, fgd_mix, fgd_outer_step(_ex) and
+ *    fgd_consensus_distance only enqueue kernels on `stream` -- no allocation, copy or
+ *    synchronisation -- so they can be recorded into a CUDA graph.  The descriptors are
+ *    kernel arguments: a graph replays the mixes it was captured with.
  */
 #ifndef FGD_H_
 #define FGD_H_

@@ -33,6 +33,7 @@ class OuterRound:
         self._x_vec2 = None   # second [P] buffer: a step that emits next round's Mix1 writes the one it does not read
         self._x_mat = None
         self._pending = None  # (event, x tensor, x_is_vector)
+        self._side_used = False   # has the side stream been given work or a wait (since capture() reset it)?
 
     # ---- Mix1: non-blocking, on the side stream ------------------------------------------
     def launch_mix1(self, mix1: MixDesc, theta_prev: torch.Tensor) -> None:
@@ -41,6 +42,7 @@ class OuterRound:
             raise ValueError("identity Mix1 needs no transfer: pass it as mix1_fused to step()")
         ready = torch.cuda.current_stream(self.device).record_event()
         self.side.wait_event(ready)
+        self._side_used = True
         if mix1.kind == FGD_MIX_MEAN:
             if self._x_vec is None:
                 self._x_vec = torch.empty(self.P, dtype=torch.float32, device=self.device)
@@ -87,8 +89,25 @@ class OuterRound:
         # the side stream may not overwrite x for the next round before this kernel has read it
         done = torch.cuda.current_stream(self.device).record_event()
         self.side.wait_event(done)
+        self._side_used = True
         if x_next is not None:
             self._pending = (done, x_next, True)
+
+    # ---- launch-bound sizes: the whole round as one CUDA graph -------------------------------
+    def capture(self, body) -> "torch.cuda.CUDAGraph":
+        """Capture ``body()`` -- calls of launch_mix1() / step() (and whatever produces theta_local)
+        on fixed buffers -- into a CUDA graph and return it; ``replay()`` then runs the round with one
+        launch from the host.  The mix descriptors are kernel arguments, so they are frozen into the
+        graph: capture one graph per distinct (Mix1, Mix2) pair of a schedule.  Run ``body()`` once
+        eagerly beforehand: the first call of a kernel sizes its launch with calls that a capture
+        does not allow, and the Mix1 result buffers must exist."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self._side_used = False
+            body()
+            if self._side_used:   # the side stream was pulled into the capture: join it back
+                torch.cuda.current_stream(self.device).wait_event(self.side.record_event())
+        return g
 
     def consensus(self, theta) -> torch.Tensor:
         fgd_consensus_distance(self.ctx, theta, self.cd_sumsq)
