@@ -138,6 +138,19 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
   if (dense) make_dense(desc, &dm);
   else if (int rc = make_gather(c, desc, &gm)) return rc;
 
+  // global average with 32 / 64 workers: several threads share a column (see mix_mean_split_kernel)
+  if (desc->kind == FGD_MIX_MEAN && (K == 32 || K == 64) && pick_vec(4, c->P, c->ld, {in, out}) == 4) {
+    const int64_t cols = 4 * kSplitBlock / (K / 16);           // columns per tile: (block / SPLIT) groups of 4, SPLIT = K / 16
+    const int64_t ntiles = (c->P + cols - 1) / cols;
+    int grid = 0;
+    auto launch = [&](auto kern) -> int {
+      if (int rc = persistent_grid(c, kern, kSplitBlock, 0, ntiles, &grid)) return rc;
+      kern<<<grid, kSplitBlock, 0, st>>>(in, out, out_is_vector ? 1 : 0, c->P, c->ld);
+      return check_launch(c, "mix_mean_split_kernel");
+    };
+    return K == 64 ? launch(mix_mean_split_kernel<64, 4, 4, kSplitBlock>) : launch(mix_mean_split_kernel<32, 2, 4, kSplitBlock>);
+  }
+
   return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
     // the averaging path keeps everything in registers: no private columns, more CTAs per SM
@@ -318,6 +331,19 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
   const int K = c->K, KT = kt_of(K);
   const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta});
   int grid = 0;
+  if ((K == 32 || K == 64) && pick_vec(4, c->P, c->ld, {theta}) == 4) {   // see consensus_split_kernel
+    auto launch = [&](auto kern, int64_t ntiles) -> int {
+      if (int r = persistent_grid(c, kern, kSplitBlock, 0, ntiles, &grid)) return r;
+      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld);
+      return check_launch(c, "consensus_split_kernel");
+    };
+    const int64_t cols = 4 * kSplitBlock / (K / 16);           // columns per tile
+    const int64_t ntiles = (c->P + cols - 1) / cols;
+    if (int r = K == 64 ? launch(consensus_split_kernel<64, 4, 4, kSplitBlock>, ntiles)
+                        : launch(consensus_split_kernel<32, 2, 4, kSplitBlock>, ntiles))
+      return r;
+    return launch_finalize(c, grid, cd_sumsq, st);
+  }
   int rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
     const size_t smem = KTc > 0 ? 0 : sizeof(float) * (size_t)K * kBlock * (VECc + 1);

@@ -17,6 +17,7 @@ using namespace fgd;  // internal header: only included by this library's own tr
 
 namespace {
 constexpr int kBlock = 128;           // threads per CTA for the column kernels
+constexpr int kSplitBlock = 256;      // threads per CTA for the kernels whose threads share a column (K = 32, 64)
 constexpr int kGradBlock = 256;
 constexpr int kMaxPartialBlocks = 148 * 16 * 2;
 }  // namespace

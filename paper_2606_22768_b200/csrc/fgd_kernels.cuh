@@ -611,6 +611,115 @@ consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials,
   }
 }
 
+// Many workers (K = 32, 64): one thread per column would hold K values and K sums, which leaves one
+// block per SM and too few loads in flight (77 % of the copy roofline at K = 64).  Here SPLIT threads
+// share a column group, each owning R = K / SPLIT rows -- the register picture of the K = 16 kernel
+// -- and exchange only their partial column sums through shared memory (double-buffered by tile
+// parity: one barrier per tile).
+template <int KT, int SPLIT, int VEC, int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ partials, int64_t P, int64_t ld) {
+  constexpr int R = KT / SPLIT;      // rows per thread
+  constexpr int G = BLOCK / SPLIT;   // column groups per tile
+  static_assert(KT % SPLIT == 0 && G % 32 == 0, "parts must be whole warps");
+  __shared__ float xs[2][SPLIT][G * VEC];
+  __shared__ double red[BLOCK / 32][R];
+  const int tid = threadIdx.x, cg = tid % G, part = tid / G, r0 = part * R;
+  float sacc[R];
+#pragma unroll
+  for (int m = 0; m < R; ++m) sacc[m] = 0.f;
+  const float invK = 1.0f / (float)KT;
+  const int64_t ntiles = (P + (int64_t)G * VEC - 1) / ((int64_t)G * VEC);
+  int it = 0;
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+    const int64_t col = (tile * G + cg) * VEC;
+    const bool live = col < P;
+    Pack<VEC> t[R];
+    Pack<VEC> sum = p_zero<VEC>();
+    if (live) {
+#pragma unroll
+      for (int m = 0; m < R; ++m) t[m] = ld_stream<VEC>(theta + (size_t)(r0 + m) * ld + col);
+#pragma unroll
+      for (int m = 0; m < R; ++m) sum = p_add<VEC>(sum, t[m]);
+    }
+    SCol<VEC>::st(xs[it & 1][part], cg, sum);
+    __syncthreads();
+    if (live) {
+      Pack<VEC> mean = SCol<VEC>::ld(xs[it & 1][0], cg);
+#pragma unroll
+      for (int q = 1; q < SPLIT; ++q) mean = p_add<VEC>(mean, SCol<VEC>::ld(xs[it & 1][q], cg));
+      mean = p_mul<VEC>(mean, invK);
+#pragma unroll
+      for (int m = 0; m < R; ++m) {
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+          const float d = t[m].v[i] - mean.v[i];
+          sq = fmaf(d, d, sq);
+        }
+        sacc[m] += sq;
+      }
+    }
+  }
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int m = 0; m < R; ++m) {
+    double d = (double)sacc[m];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
+    if (lane == 0) red[warp][m] = d;
+  }
+  __syncthreads();
+  if (tid < KT) {                    // worker tid = rows of part tid / R, summed over that part's warps
+    const int q = tid / R, j = tid % R;
+    double d = 0.0;
+#pragma unroll
+    for (int w = 0; w < G / 32; ++w) d += red[q * (G / 32) + w][j];
+    partials[(size_t)blockIdx.x * KT + tid] = d;
+  }
+}
+
+// Global average with many workers, same split: out = column mean as one row (out_is_vector) or
+// written to every row.
+template <int KT, int SPLIT, int VEC, int BLOCK>
+__global__ void __launch_bounds__(BLOCK)
+mix_mean_split_kernel(const float* __restrict__ in, float* __restrict__ out, int out_is_vector, int64_t P, int64_t ld) {
+  constexpr int R = KT / SPLIT;
+  constexpr int G = BLOCK / SPLIT;
+  static_assert(KT % SPLIT == 0 && G % 32 == 0, "parts must be whole warps");
+  __shared__ float xs[2][SPLIT][G * VEC];
+  const int tid = threadIdx.x, cg = tid % G, part = tid / G, r0 = part * R;
+  const float invK = 1.0f / (float)KT;
+  const int64_t ntiles = (P + (int64_t)G * VEC - 1) / ((int64_t)G * VEC);
+  int it = 0;
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+    const int64_t col = (tile * G + cg) * VEC;
+    const bool live = col < P;
+    Pack<VEC> sum = p_zero<VEC>();
+    if (live) {
+      Pack<VEC> t[R];
+#pragma unroll
+      for (int m = 0; m < R; ++m) t[m] = ld_stream<VEC>(in + (size_t)(r0 + m) * ld + col);
+#pragma unroll
+      for (int m = 0; m < R; ++m) sum = p_add<VEC>(sum, t[m]);
+    }
+    SCol<VEC>::st(xs[it & 1][part], cg, sum);
+    __syncthreads();
+    if (live && (!out_is_vector || part == 0)) {
+      Pack<VEC> mean = SCol<VEC>::ld(xs[it & 1][0], cg);
+#pragma unroll
+      for (int q = 1; q < SPLIT; ++q) mean = p_add<VEC>(mean, SCol<VEC>::ld(xs[it & 1][q], cg));
+      mean = p_mul<VEC>(mean, invK);
+      if (out_is_vector) {
+        st_stream<VEC>(out + col, mean);
+      } else {
+#pragma unroll
+        for (int m = 0; m < R; ++m) st_stream<VEC>(out + (size_t)(r0 + m) * ld + col, mean);
+      }
+    }
+  }
+}
+
 // out[m] = sum_b partials[b][m], fixed order: one warp per worker, lanes stride the blocks,
 // then a shuffle tree.  Deterministic.
 static __global__ void __launch_bounds__(32)

@@ -53,6 +53,7 @@ MIX_CASES = [
     (32, 20002, ("hypercube", 0.1)), (64, 10000, ("dense", SINK64)), (64, 4097, ("ring",)),
     (16, 8192, ("dense", gen.sinkhorn_W(1, 16))), (7, 2048, ("dense", gen.sinkhorn_W(2, 7))),
     (2, 1000, ("ring",)), (1, 100, ("identity",)), (8, 1000, ("identity",)),
+    (64, 70004, ("mean",)), (32, 50000, ("mean",)), (64, 30001, ("mean",)),   # threads share a column (and its fall-back)
 ]
 
 
@@ -74,7 +75,7 @@ def test_mix_matrix_output(K, P, spec):
     assert torch.equal(f_in[:, :P], out)
 
 
-@pytest.mark.parametrize("K,P", [(4, 1 << 20), (16, 30001), (6, 513), (64, 4096)])
+@pytest.mark.parametrize("K,P", [(4, 1 << 20), (16, 30001), (6, 513), (64, 4096), (64, 100004), (32, 65540), (32, 999)])
 def test_mix_mean_vector_output(K, P):
     x = gen.theta0(4, K, P, 0.02, 5e-3)
     f_in, _ = upload(x, P)
@@ -88,7 +89,8 @@ def test_mix_mean_vector_output(K, P):
 
 # ------------------------------------------------------------------ fgd_consensus_distance
 @pytest.mark.parametrize("K,P,ld", [(4, 1 << 20, None), (16, 100001, 100004), (64, 20000, 20000), (32, 30002, 30002),
-                                     (5, 7777, 7780), (1, 50, 50), (2, 3, 4)])
+                                     (5, 7777, 7780), (1, 50, 50), (2, 3, 4), (64, 150004, 150016), (32, 200000, 200000),
+                                     (64, 131, 132), (32, 4, 4)])
 def test_consensus_distance(K, P, ld):
     ld = P if ld is None else ld
     th = gen.theta0(5, K, P, 0.02, 7e-4)
