@@ -162,9 +162,23 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
       if (int rc = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return rc;
       kern<<<grid, kBlock, smem, st>>>(a, dm);
     } else {
-      auto kern = mix_kernel<KTc, VECc, false, kBlock, GatherMix>;
-      if (int rc = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return rc;
-      kern<<<grid, kBlock, smem, st>>>(a, gm);
+      auto launch = [&](auto kern) -> int {
+        if (int rc = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return rc;
+        kern<<<grid, kBlock, smem, st>>>(a, gm);
+        return FGD_OK;
+      };
+      int rc = FGD_OK;
+      // compile-time worker counts also get a compile-time neighbour count (fully unrolled gathers)
+      const int dt = (KTc > 0 && gm.kind == KMIX_GATHER && (gm.D == 1 || gm.D == 2 || gm.D == 4)) ? gm.D : -1;
+      if constexpr (KTc > 0) {
+        if (dt == 1) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 1>);
+        else if (dt == 2) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 2>);
+        else if (dt == 4) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 4>);
+        else rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix>);
+      } else {
+        rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix>);
+      }
+      if (rc) return rc;
     }
     return check_launch(c, "mix_kernel");
   });

@@ -455,7 +455,8 @@ struct MixArgs {
   int out_is_vector;
 };
 
-template <int KT, int VEC, bool DENSE, int BLOCK, typename MX>
+// DT: compile-time neighbour slot count of a sparse mix (-1 = read at run time), see gather_row.
+template <int KT, int VEC, bool DENSE, int BLOCK, typename MX, int DT = -1>
 __global__ void __launch_bounds__(BLOCK) mix_kernel(const MixArgs a, const MX mx) {
   extern __shared__ __align__(16) float smem[];
   const int K = KT > 0 ? KT : a.K;
@@ -514,7 +515,7 @@ __global__ void __launch_bounds__(BLOCK) mix_kernel(const MixArgs a, const MX mx
     } else {
 #pragma unroll(KT > 0 ? KT : 2)
       for (int m = 0; m < K; ++m)
-        st_stream<VEC>(a.out + (size_t)m * ld + col, gather_row<VEC, BLOCK>(mx, m, cs, tid));
+        st_stream<VEC>(a.out + (size_t)m * ld + col, gather_row<VEC, BLOCK, DT>(mx, m, cs, tid));
     }
   }
 }
