@@ -140,6 +140,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_slot;
   __shared__ float xchg[2][T];       // the two halves of a column exchange their theta_new sums
+  __shared__ float xsum[2][T];       // ... and, for a fused global-average Mix1, their theta_prev sums
 
   const StepArgs& a = ta.s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -261,10 +262,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           g[n] = tp - B[(r0 + n) * T + c];
           tsum += tp;
         }
-        if (need_tsum) {                           // the column mean needs the other half too
-#pragma unroll
-          for (int n = 0; n < H; ++n) tsum += A[((H - r0) + n) * T + c];
-        }
+        if (need_tsum) xsum[h][c] = tsum;          // the column mean needs the other half's sum too
         if constexpr (XM == 2) {                   // gossip Mix1 of this thread's rows, from the stage
           const int D1 = m1.D;                     // (uniform) -> a fully unrolled gather per slot count
           if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, xr);
@@ -279,6 +277,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       }
       named_bar_sync(1, CONS);                    // every consumer has read its theta_prev / theta_local
       if (*(volatile int*)&abort_flag) break;     // uniform: the flag was written before the barrier
+      if (need_tsum) tsum += xsum[h ^ 1][c];
       // ---- operands: g_hi over the theta_local box, g_lo over the theta_prev box
 #pragma unroll
       for (int n = 0; n < H; n += 4) {

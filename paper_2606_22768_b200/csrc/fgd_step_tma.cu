@@ -21,7 +21,7 @@ bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, con
   if (!c->encode_tiled || a.n_ranges != 0) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
-  return (size_t)c->max_smem_optin >= TcShape<kTcMaxK>::kSmem + 2048;
+  return (size_t)c->max_smem_optin >= TcShape<kTcMaxK>::kSmem + 2304;   // + static shared memory (barriers, exchange rows)
 }
 
 template <int KP>
