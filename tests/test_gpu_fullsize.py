@@ -41,16 +41,16 @@ def _spec(cfg, which):
     kind = cfg[which][0]
     if kind == "dense":
         return ("dense", gen.sinkhorn_W(0, cfg["K"]))
-    if cfg["p_fail"] > 0 and kind in ("ring", "xor", "hypercube"):
+    if cfg["p_fail"] > 0 and kind in ("ring", "xor", "hypercube", "matching"):
         return (kind, cfg["p_fail"], fgd.FGD_RENORM_METROPOLIS)
     return (kind,)
 
 
-@pytest.mark.parametrize("cfg_id,rounds", [(2, 10), (3, 10), (4, 20), (5, 5)])
+@pytest.mark.parametrize("cfg_id,rounds", [(2, 10), (3, 10), (4, 20), (5, 5), (6, 3)])
 def test_full_size_config(cfg_id, rounds):
     cfg = bench.CONFIGS[cfg_id]
     K, P, seed = cfg["K"], cfg["P"], 0
-    need = (4 if cfg["mix1"][0] != "mean" else 3) * K * P * 4 + (1 << 30)
+    need = (4 if cfg["mix1"][0] != "mean" else 3) * K * P * 4 + 4 * P + (2 << 30)
     if torch.cuda.mem_get_info()[0] < need:
         pytest.skip("not enough free HBM for this configuration")
     sig = (gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1]
