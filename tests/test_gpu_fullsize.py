@@ -90,6 +90,13 @@ def test_full_size_config(cfg_id, rounds):
             assert_param_close(theta[:, p0:p0 + WIDTH], o_theta[p0], f"cfg{cfg_id} round {r} theta_new block {p0}")
             assert_param_close(mom[:, p0:p0 + WIDTH], o_v[p0], f"cfg{cfg_id} round {r} momentum block {p0}")
     fgd.fgd_device_status(drv.ctx)
+    if cfg_id == 2:
+        # the fused consensus sums of the last round against the oracle over ALL columns (columns are
+        # independent, so the oracle takes them in chunks and the per-worker sums add up)
+        total = np.zeros(K)
+        for c0 in range(0, P, 1 << 24):
+            total += oracle.consensus_sumsq(theta[:, c0:min(P, c0 + (1 << 24))].cpu().numpy())
+        assert_cd_close(drv.cd_sumsq, total, P, "cfg2 fused consensus sums, all columns")
     # a stand-alone consensus call on a sampled window (row stride P, 16-byte aligned start)
     p0 = blocks[len(blocks) // 2] // 4 * 4
     win = fgd.Context(K, WIDTH, P)
