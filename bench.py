@@ -72,6 +72,8 @@ def parse_args():
     ap.add_argument("--average-momentum", action="store_true", help="variant: GlobalM1S (needs Mix1 = mean)")
     ap.add_argument("--chain-mix1", action="store_true",
                     help="variant: the fused step also writes next round's global-average Mix1 (no Mix1 kernel)")
+    ap.add_argument("--fuse-mix1", action="store_true",
+                    help="variant: Mix1 computed inside the fused step from the staged theta_prev (one launch per round, 20 B per worker-parameter)")
     ap.add_argument("--graph", action="store_true",
                     help="variant: capture the round (Mix1 + fused step) into one CUDA graph and time its replays")
     ap.add_argument("--kernels", action="store_true",
@@ -281,11 +283,23 @@ def run_ours(args):
         cfg["name"] += " [variant: momentum averaged (GlobalM1S)]"
     if args.chain_mix1:
         cfg["name"] += " [variant: Mix1 (mean) of round r+1 emitted by the fused step of round r]"
+    if args.fuse_mix1:
+        if args.chain_mix1 or args.graph or cfg["mix1"][0] == "dense":
+            raise SystemExit("--fuse-mix1 excludes --chain-mix1 / --graph and needs a mean or sparse Mix1")
+        cfg["name"] += " [variant: Mix1 fused into the step kernel]"
 
     def one_round(r, ev_pair=None):
         m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
         m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
         drv.cd_sumsq = cd_log[r]
+        if args.fuse_mix1:
+            if ev_pair is not None:
+                ev_pair[0].record(main)
+            drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix1_fused=m1, mix2_ranges=ranges,
+                     average_momentum=args.average_momentum)
+            if ev_pair is not None:
+                ev_pair[1].record(main)
+            return
         if not (args.chain_mix1 and drv._pending is not None):
             drv.launch_mix1(m1, theta)
         if ev_pair is not None:
@@ -345,6 +359,8 @@ def run_ours(args):
     x_vec = cfg["mix1"][0] == "mean"
     step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
     mix1_bytes = (4 * K * P + 4 * P) if x_vec else 8 * K * P
+    if args.fuse_mix1:
+        step_bytes, mix1_bytes = 20 * K * P, 0
     peak, peak_kind = measured_peak()
     achieved = step_bytes / (kern_ms * 1e-3) / 1e9
     tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
