@@ -125,7 +125,9 @@ __device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A,
 // problem is zero-padded to KP: the TMA boxes stay KP rows tall (rows at or beyond KR are outside
 // the tensor and arrive as zeros without touching HBM), W is padded with zero rows and columns,
 // and only the first KR rows are stored.
-template <int KP, int XM, bool FULL>
+// SUB: Mix2 only on the columns inside the caller's ranges, the identity elsewhere (the thread keeps
+// its g values in registers across the MMA and takes them instead of the accumulator row there).
+template <int KP, int XM, bool FULL, bool SUB = false>
 __global__ void __launch_bounds__(kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
@@ -334,6 +336,12 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
       tmem_ld_cols<H>(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
+      if constexpr (SUB) {
+        if (!mix2_applies(a, col)) {
+#pragma unroll
+          for (int m = 0; m < H; ++m) gh[m] = g[m];
+        }
+      }
       // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
       float asum = 0.f;
       if (live) {

@@ -18,7 +18,10 @@ bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, con
   const int K = c->K;
   if (K > kTcMaxK || K < kTcMinK) return false;
   if (kt_of(K) == 16 || (kt_of(K) == 32 && !really_dense)) return false;
-  if (!c->encode_tiled || a.n_ranges != 0) return false;
+  if (!c->encode_tiled) return false;
+  // column-range Mix2 is built for the one-value-per-column Mix1 (the "-subset" configurations pair it
+  // with the global average)
+  if (a.n_ranges != 0 && !(a.xsrc == XSRC_VECTOR || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_MEAN))) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   return (size_t)c->max_smem_optin >= TcShape<kTcMaxK>::kSmem + 2304;   // + static shared memory (barriers, exchange rows)
@@ -46,7 +49,10 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
   switch (xm) {
     case 1: return full ? launch(outer_step_dense_tc_kernel<KP, 1, true>) : launch(outer_step_dense_tc_kernel<KP, 1, false>);
     case 2: return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
-    default: return full ? launch(outer_step_dense_tc_kernel<KP, 0, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false>);
+    default:
+      if (a.n_ranges != 0)
+        return full ? launch(outer_step_dense_tc_kernel<KP, 0, true, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false, true>);
+      return full ? launch(outer_step_dense_tc_kernel<KP, 0, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false>);
   }
 }
 

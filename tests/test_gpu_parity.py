@@ -321,6 +321,8 @@ VARIANTS = [
     ("dense16-subset", 16, 8000, ("ring",), ("dense", gen.sinkhorn_W(1, 16)), True, False),
     ("dense48-GlobalM1S", 48, 5000, ("mean",), ("dense", gen.sinkhorn_W(3, 48)), False, True),
     ("ring40-GlobalM1S", 40, 4001, ("mean",), ("ring",), False, True),
+    ("dense48-subset", 48, 6000, ("mean",), ("dense", gen.sinkhorn_W(3, 48)), True, False),
+    ("ring24-subset-GlobalM1S", 24, 9000, ("mean",), ("ring",), True, True),
 ]
 
 
