@@ -151,6 +151,20 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
     return K == 64 ? launch(mix_mean_split_kernel<64, 4, 4, kSplitBlock>) : launch(mix_mean_split_kernel<32, 2, 4, kSplitBlock>);
   }
 
+  // worker counts above 16 without a compile-time fp32 kernel, and dense matrices from K = 32 up:
+  // the tensor-core kernel (any mix is a dense matrix, so a sparse or mean one is densified for it)
+  if (!out_is_vector && (c->path == FGD_PATH_AUTO || c->path == FGD_PATH_TMA) && fgd_mix_tc_eligible(c, in, dense)) {
+    bool ok = true;
+    if (!dense) {
+      double Wd[FGD_MAX_K * FGD_MAX_K];
+      ok = fgd_dense_matrix(desc, Wd) == FGD_OK;
+      if (ok)
+        for (int m = 0; m < K; ++m)
+          for (int n = 0; n < K; ++n) dm.Wt[n * K + m] = (float)Wd[m * K + n];
+    }
+    if (ok) return fgd_launch_mix_dense_tc(c, in, out, dm, st);
+  }
+
   return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
     // the averaging path keeps everything in registers: no private columns, more CTAs per SM

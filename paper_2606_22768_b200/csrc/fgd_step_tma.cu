@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include "fgd_mix_dense_tc.cuh"
 #include "fgd_step_dense_tc.cuh"
 #include "fgd_tma_host.h"
 
@@ -70,6 +71,41 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   }
   if (rc) return rc;
   return check_launch(c, "outer_step_dense_tc_kernel");
+}
+
+// Stand-alone mix on the tensor cores: same worker counts as the step (K = 32 only for a really
+// dense matrix: its sparse fp32 kernel is at the copy roofline already).
+bool fgd_mix_tc_eligible(const fgd_ctx* c, const float* in, bool really_dense) {
+  const int K = c->K;
+  if (K > kTcMaxK || K < kTcMinK || kt_of(K) == 16 || (kt_of(K) == 32 && !really_dense)) return false;
+  if (!c->encode_tiled || c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096 || !aligned16(in)) return false;
+  return (size_t)c->max_smem_optin >= TcMixShape<kTcMaxK>::kSmem + 256;
+}
+
+template <int KP>
+static int launch_mix_tc(fgd_ctx* c, const TcMixArgs& a, const DenseMix& dm, cudaStream_t st) {
+  CUtensorMap tin;
+  if (int rc = make_tensor_map(c, &tin, a.in, kTcCols, KP)) return rc;
+  const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
+  int grid = 0;
+  auto launch = [&](auto kern) -> int {
+    if (int r = persistent_grid(c, kern, kTcConsumers + 32, TcMixShape<KP>::kSmem, ntiles, &grid)) return r;
+    kern<<<grid, kTcConsumers + 32, TcMixShape<KP>::kSmem, st>>>(a, dm, tin);
+    return FGD_OK;
+  };
+  return c->K == KP ? launch(mix_dense_tc_kernel<KP, true>) : launch(mix_dense_tc_kernel<KP, false>);
+}
+
+int fgd_launch_mix_dense_tc(fgd_ctx* c, const float* in, float* out, const DenseMix& dm, cudaStream_t st) {
+  const TcMixArgs a{in, out, c->P, c->ld, c->K, c->status};
+  int rc = FGD_OK;
+  switch (tc_padded_k(c->K)) {
+    case 32: rc = launch_mix_tc<32>(c, a, dm, st); break;
+    case 48: rc = launch_mix_tc<48>(c, a, dm, st); break;
+    default: rc = launch_mix_tc<64>(c, a, dm, st); break;
+  }
+  if (rc) return rc;
+  return check_launch(c, "mix_dense_tc_kernel");
 }
 
 bool fgd_tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, FgdTmaShape* out) {

@@ -54,6 +54,10 @@ MIX_CASES = [
     (16, 8192, ("dense", gen.sinkhorn_W(1, 16))), (7, 2048, ("dense", gen.sinkhorn_W(2, 7))),
     (2, 1000, ("ring",)), (1, 100, ("identity",)), (8, 1000, ("identity",)),
     (64, 70004, ("mean",)), (32, 50000, ("mean",)), (64, 30001, ("mean",)),   # threads share a column (and its fall-back)
+    # tensor-core mix: worker counts 17..64 (zero-padded to 32 / 48 / 64), sparse mixes densified
+    (48, 9001, ("ring",)), (40, 5000, ("dense", gen.sinkhorn_W(8, 40))), (33, 4100, ("matching",)), (63, 3000, ("mean",)),
+    (32, 6002, ("dense", gen.sinkhorn_W(7, 32))), (24, 7000, ("ring", 0.3)), (17, 2000, ("dense", gen.sinkhorn_W(9, 17))),
+    (64, 20000, ("hypercube", 0.1)),
 ]
 
 
