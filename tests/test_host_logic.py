@@ -146,3 +146,49 @@ def test_gpu_entry_points_fail_loudly_without_a_device():
     with pytest.raises(fgd.FgdError) as e:
         fgd.Context(4, 128)
     assert e.value.status == fgd.FGD_ERR_CUDA
+
+
+def _random_graph(rng, K, max_deg):
+    """Random undirected graph as padded neighbour lists (-1 = empty slot), Metropolis base weights."""
+    adj = [[] for _ in range(K)]
+    pairs = [(a, b) for a in range(K) for b in range(a + 1, K)]
+    rng.shuffle(pairs)
+    for a, b in pairs:
+        if len(adj[a]) < max_deg and len(adj[b]) < max_deg and rng.random() < 0.5:
+            adj[a].append(b)
+            adj[b].append(a)
+    D = max(1, max(len(r) for r in adj))
+    nbr = [r + [-1] * (D - len(r)) for r in adj]
+    deg = [len(r) for r in adj]
+    w = [[(1.0 / (1 + max(deg[m], deg[n])) if n >= 0 else 0.0) for n in nbr[m]] for m in range(K)]
+    ws = [1.0 - sum(w[m]) for m in range(K)]
+    return nbr, w, ws
+
+
+@pytest.mark.parametrize("renorm", [fgd.FGD_RENORM_NONE, fgd.FGD_RENORM_SELF_ABSORB, fgd.FGD_RENORM_METROPOLIS])
+def test_masks_and_renormalisation_on_random_graphs(renorm):
+    """Irregular degrees, empty slots, every drop rate: the two implementations agree (masks bit for
+    bit, weights to 1e-7) and the invariants of the reading hold -- symmetric, non-negative, and
+    doubly stochastic under both renormalisation rules."""
+    rng = np.random.default_rng(2024)
+    for trial in range(40):
+        K = int(rng.integers(3, 65))
+        nbr, w, ws = _random_graph(rng, K, int(rng.integers(1, fgd.FGD_MAX_D + 1)))
+        p_fail = float(rng.choice([0.0, 0.05, 0.3, 0.7, 1.0]))
+        nbr_np = np.array(nbr, dtype=np.int32)
+        mask = T.edge_mask(trial, 3 * trial, 1 + trial % 2, p_fail, nbr)
+        assert fgd.fgd_edge_mask(trial, 3 * trial, 1 + trial % 2, p_fail, nbr_np).tolist() == mask
+        desc = fgd.MixDesc.sparse(nbr, w, ws, mask, renorm)
+        w_eff, ws_eff = fgd.fgd_effective_weights(desc)
+        w32 = np.array(w, dtype=np.float32).astype(np.float64).tolist()
+        ws32 = np.array(ws, dtype=np.float32).astype(np.float64).tolist()
+        ref_w, ref_ws = T.effective_weights(nbr, w32, ws32, mask, renorm)
+        np.testing.assert_allclose(w_eff, np.array(ref_w), rtol=0, atol=1e-7)
+        np.testing.assert_allclose(ws_eff, np.array(ref_ws), rtol=0, atol=1e-7)
+        W = fgd.fgd_dense_matrix(desc)
+        assert np.array_equal(W, W.T) and (W >= -1e-7).all()
+        if renorm != fgd.FGD_RENORM_NONE:
+            np.testing.assert_allclose(W.sum(0), 1.0, rtol=0, atol=4e-7)
+            np.testing.assert_allclose(W.sum(1), 1.0, rtol=0, atol=4e-7)
+        if p_fail == 1.0 and renorm != fgd.FGD_RENORM_NONE:
+            np.testing.assert_allclose(W, np.eye(K), rtol=0, atol=4e-7)     # every exchange failed: nobody mixes
