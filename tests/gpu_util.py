@@ -63,6 +63,32 @@ def make_mix(spec, K, rnd, seed, mix_id):
             assert d.edge_mask.tolist() == mask
         w_eff, ws_eff = T.effective_weights(nbr, w32, ws32, mask, renorm if mask is not None else T.RENORM_NONE)
         return d, np.array(T.dense_from_sparse(nbr, w_eff, ws_eff), dtype=np.float64)
+    if kind == "randgraph":   # seeded irregular graph: degrees 0..max_deg, empty slots, Metropolis base weights
+        max_deg = spec[1]
+        p_fail = spec[2] if len(spec) > 2 else 0.0
+        rng = np.random.default_rng(1000 * K + max_deg)
+        adj = [[] for _ in range(K)]
+        pairs = [(a, b) for a in range(K) for b in range(a + 1, K)]
+        rng.shuffle(pairs)
+        for a, b in pairs:
+            if len(adj[a]) < max_deg and len(adj[b]) < max_deg and rng.random() < 0.6:
+                adj[a].append(b)
+                adj[b].append(a)
+        D = max(1, max(len(r) for r in adj))
+        nbr = [r + [-1] * (D - len(r)) for r in adj]
+        deg = [len(r) for r in adj]
+        w = [[(1.0 / (1 + max(deg[m], deg[n])) if n >= 0 else 0.0) for n in nbr[m]] for m in range(K)]
+        ws = [1.0 - sum(w[m]) for m in range(K)]
+        d = fgd.MixDesc.sparse(nbr, w, ws)
+        w32 = np.array(w, dtype=np.float32).astype(np.float64).tolist()
+        ws32 = np.array(ws, dtype=np.float32).astype(np.float64).tolist()
+        mask = None
+        if p_fail > 0.0:
+            d = d.with_failures(seed, rnd, mix_id, p_fail, fgd.FGD_RENORM_METROPOLIS)
+            mask = T.edge_mask(seed, rnd, mix_id, p_fail, nbr)
+            assert d.edge_mask.tolist() == mask
+        w_eff, ws_eff = T.effective_weights(nbr, w32, ws32, mask, T.RENORM_METROPOLIS if mask is not None else T.RENORM_NONE)
+        return d, np.array(T.dense_from_sparse(nbr, w_eff, ws_eff), dtype=np.float64)
     if kind == "isolated":    # a sparse descriptor with no neighbour slots at all (D = 0): W = I
         d = fgd.MixDesc.sparse(np.zeros((K, 0), dtype=np.int32), np.zeros((K, 0), dtype=np.float32), np.ones(K, dtype=np.float32))
         return d, oracle.dense_W("identity", K)

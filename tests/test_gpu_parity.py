@@ -57,7 +57,7 @@ MIX_CASES = [
     # tensor-core mix: worker counts 17..64 (zero-padded to 32 / 48 / 64), sparse mixes densified
     (48, 9001, ("ring",)), (40, 5000, ("dense", gen.sinkhorn_W(8, 40))), (33, 4100, ("matching",)), (63, 3000, ("mean",)),
     (32, 6002, ("dense", gen.sinkhorn_W(7, 32))), (24, 7000, ("ring", 0.3)), (17, 2000, ("dense", gen.sinkhorn_W(9, 17))),
-    (64, 20000, ("hypercube", 0.1)),
+    (64, 20000, ("hypercube", 0.1)), (16, 9000, ("randgraph", 5, 0.2)), (40, 3000, ("randgraph", 3)), (7, 2000, ("randgraph", 2)),
 ]
 
 
@@ -155,6 +155,11 @@ STEP_CASES = [
     (64, 3000, ("identity",), ("ring",)),
     (32, 6000, ("matching",), ("dense", gen.sinkhorn_W(7, 32))),
     (56, 3001, ("circulant", 4, 0.2), ("circulant", 3)),
+    # irregular graphs: uneven degrees, empty slots, odd slot counts
+    (12, 5000, ("randgraph", 3), ("randgraph", 5, 0.2)),
+    (16, 6001, ("randgraph", 5, 0.1), ("randgraph", 3)),
+    (48, 4000, ("randgraph", 7), ("randgraph", 7, 0.3)),
+    (64, 3000, ("randgraph", 3, 0.2), ("randgraph", 6)),
 ]
 
 
