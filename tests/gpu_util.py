@@ -32,8 +32,12 @@ def assert_cd_close(got, ref, P, what=""):
     got = got.detach().cpu().numpy() if isinstance(got, torch.Tensor) else np.asarray(got)
     ref = np.asarray(ref, dtype=np.float64)
     floor = 1e-12 * P  # exact-consensus cases: fp32 means of equal values are off by an ulp
+    # theta_new and the column mean are each rounded to fp32 (a few ulps of |theta| <= 0.1, delta <= 8e-9)
+    # before the deviation d is squared: s moves by about 2 delta sqrt(s) (random signs), which only
+    # matters when there are so few columns that nothing averages out; 4 sigma of that.
+    rounding = 8 * 8e-9 * np.sqrt(np.abs(ref))
     err = np.abs(got - ref)
-    assert ((err <= CD_RTOL * np.abs(ref)) | (err <= floor)).all(), f"{what}: got {got} ref {ref}"
+    assert ((err <= CD_RTOL * np.abs(ref)) | (err <= floor) | (err <= rounding)).all(), f"{what}: got {got} ref {ref}"
 
 
 def make_mix(spec, K, rnd, seed, mix_id):

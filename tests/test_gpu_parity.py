@@ -155,6 +155,12 @@ STEP_CASES = [
     (64, 3000, ("identity",), ("ring",)),
     (32, 6000, ("matching",), ("dense", gen.sinkhorn_W(7, 32))),
     (56, 3001, ("circulant", 4, 0.2), ("circulant", 3)),
+    # fewer columns than one tile (and than one vector)
+    (64, 5, ("mean",), ("dense", SINK64)),
+    (48, 1, ("mean",), ("ring",)),
+    (16, 3, ("mean",), ("ring",)),
+    (8, 130, ("ring",), ("xor",)),
+    (3, 2, ("mean",), ("ring",)),
     # irregular graphs: uneven degrees, empty slots, odd slot counts
     (12, 5000, ("randgraph", 3), ("randgraph", 5, 0.2)),
     (16, 6001, ("randgraph", 5, 0.1), ("randgraph", 3)),
