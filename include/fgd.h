@@ -77,12 +77,16 @@ int fgd_destroy(fgd_ctx* ctx);
  * last failing fgd_create / host helper on this thread.  The string is owned by the library. */
 const char* fgd_last_error(const fgd_ctx* ctx);
 const char* fgd_status_string(int status);
-/* Which kernel family fgd_outer_step uses.  AUTO (default): a TMA-pipelined kernel when the
- * tensors allow it (16-byte aligned bases, ld % 4 == 0, two pipeline stages fit in shared
- * memory), else the register kernel; a dense Mix2 with K = 64 runs its contraction on the
- * tensor cores (3 x TF32, fp32 accumulate) when Mix1 is the mean.  REGISTER / TMA force a
- * family (TMA fails with FGD_ERR_UNSUPPORTED when not eligible); TMA_FP32 is TMA with the
- * dense contraction kept on the fp32 CUDA cores.  All compute the same round. */
+/* Which kernel family fgd_outer_step and fgd_mix use.  AUTO (default): a TMA-pipelined kernel
+ * when the tensors allow it (16-byte aligned bases, ld % 4 == 0, fewer than 2^31 - 4096
+ * columns, two pipeline stages fit in shared memory), else the register kernel.  Within the
+ * TMA family, K = 64, every K in [17, 63] other than 32, and a dense matrix at K = 32 run the
+ * mix as a tensor-core contraction (3 x TF32 split, fp32 accumulate: relative error about
+ * 2^-22 instead of fp32's 2^-24; sparse and mean mixes are densified for it); K = 2, 4, 8, 16,
+ * 32 with sparse or mean mixes run compile-time fp32 kernels, other K below 17 a run-time-K
+ * fp32 kernel.  REGISTER / TMA force a family (TMA fails with FGD_ERR_UNSUPPORTED when not
+ * eligible); TMA_FP32 is the TMA family with every contraction kept on the fp32 CUDA cores.
+ * All compute the same round. */
 typedef enum { FGD_PATH_AUTO = 0, FGD_PATH_REGISTER = 1, FGD_PATH_TMA = 2, FGD_PATH_TMA_FP32 = 3 } fgd_path;
 int fgd_set_path(fgd_ctx* ctx, int path);
 /* Synchronises `stream` and reports whether any kernel of this context abandoned a bounded
