@@ -127,8 +127,14 @@ __device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A,
 // and only the first KR rows are stored.
 // SUB: Mix2 only on the columns inside the caller's ranges, the identity elsewhere (the thread keeps
 // its g values in registers across the MMA and takes them instead of the accumulator row there).
-template <int KP, int XM, bool FULL, bool SUB = false>
-__global__ void __launch_bounds__(kTcConsumers + 32)
+// NG: consumer groups.  With two, group g takes every second tile of the CTA (its own stages,
+// named barriers, MMA barrier and accumulator columns), so one group's epilogue -- TMEM read,
+// update, stores -- overlaps the other's operand preparation and MMA.  544 threads leave 96
+// registers each: that fits the 32-worker shape (measured: K = 17 3.3 -> 4.7 TB/s, K = 24 4.6 ->
+// 5.7, dense K = 32 5.4 -> 5.6) and spills at 48 and 64 workers (K = 64: 10.8 -> 13.8 ms), which
+// therefore keep one group.
+template <int KP, int XM, bool FULL, bool SUB = false, int NG = 1>
+__global__ void __launch_bounds__(NG * kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                            const __grid_constant__ CUtensorMap tm_mom, const __grid_constant__ CUtensorMap tm_x) {
@@ -136,21 +142,26 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   constexpr bool XMAT = XM != 0;                    // x differs from row to row
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
   constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
+  constexpr int ALLC = NG * CONS;                   // all consumer threads; the producer warp follows them
+  static_assert(STAGES % NG == 0, "every stage belongs to one group");
   const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];   // full[], empty[], mma
+  __shared__ __align__(8) unsigned long long bars[2 * STAGES + NG];  // full[], empty[], mma[group]
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_slot;
-  __shared__ float xchg[2][T];       // the two halves of a column exchange their theta_new sums
-  __shared__ float xsum[2][T];       // ... and, for a fused global-average Mix1, their theta_prev sums
+  __shared__ float xchg[NG][2][T];   // the two halves of a column exchange their theta_new sums
+  // ... and, for a fused global-average Mix1, their theta_prev sums
+  __shared__ float xsum[NG][2][T];
+  static_assert(NG == 1 || KP < 64, "two groups at 64 workers: no shared memory left for the exchange rows (and no registers)");
 
   const StepArgs& a = ta.s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gid = (NG > 1 && tid < ALLC) ? tid / CONS : 0;      // consumer group of this thread
   const bool want_cd = a.partials != nullptr;
   unsigned char* base = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);   // TMA wants 128-byte alignment
   unsigned char* wb_hi = base + (size_t)STAGES * 3 * kTcBox;
   unsigned char* wb_lo = wb_hi + kTcWBytes;
-  const uint32_t mma_bar = smem_u32(&bars[2 * STAGES]);
+  const uint32_t mma_bar = smem_u32(&bars[2 * STAGES + gid]);
 
   const int64_t P = a.P, ld = a.ld;
   const int64_t ntiles = (P + T - 1) / T;
@@ -161,12 +172,12 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       mbar_init(smem_u32(&bars[s]), 1);
       mbar_init(smem_u32(&bars[STAGES + s]), CONS);
     }
-    mbar_init(mma_bar, 1);
+    for (int g = 0; g < NG; ++g) mbar_init(smem_u32(&bars[2 * STAGES + g]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // B operand = W^T as an N x K (m x n) matrix, K-major, no swizzle: 8-row x 16-byte core
   // matrices; core matrices adjacent in K are 128 B apart, adjacent in N SBO = 32 K bytes apart.
-  for (int i = tid; i < K * K; i += CONS + 32) {
+  for (int i = tid; i < K * K; i += ALLC + 32) {
     const int n = i / K, m = i % K;          // m2.Wt[n*KR+m] = W[m][n]
     const float w = (FULL || (n < KR && m < KR)) ? m2.Wt[n * KR + m] : 0.f;
     const float hi = to_tf32(w);
@@ -174,8 +185,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     *reinterpret_cast<float*>(wb_hi + off) = hi;
     *reinterpret_cast<float*>(wb_lo + off) = w - hi;
   }
-  if (warp == CONS / 32) {   // the producer warp owns tensor memory: allocate the accumulator columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)Shape::kTmemCols) : "memory");
+  if (warp == ALLC / 32) {   // the producer warp owns tensor memory: allocate the accumulator columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(NG * Shape::kTmemCols)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // W operands are read by the MMA (async proxy)
@@ -183,12 +194,13 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t tmem_acc = tmem_base + (uint32_t)(gid * Shape::kTmemCols);   // this group's accumulator columns
 
   float sacc[H];
 #pragma unroll
   for (int m = 0; m < H; ++m) sacc[m] = 0.f;
 
-  if (warp == CONS / 32) {
+  if (warp == ALLC / 32) {
     // ===================================================== producer (one elected lane)
     if (lane == 0) {
       uint64_t policy;
@@ -222,7 +234,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     // Two threads per column: thread (c, h) owns column c of the tile and the workers
     // [H h, H h + H), H = K / 2 -- eight consumer warps instead of four hide the shared-memory,
     // TMEM and barrier latencies, and half-length arrays keep everything in registers.
-    const int c = tid & (T - 1), h = tid >> 7, r0 = h * H;
+    const int lt = tid & (CONS - 1);              // index within the group
+    const int c = lt & (T - 1), h = lt >> 7, r0 = h * H;
     const float invK = 1.0f / (float)KR;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
     const float lr = a.lr, mu = a.mu;
@@ -233,8 +246,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     const uint32_t op_row = (uint32_t)(c >> 3) * SBO + (uint32_t)(c & 7) * 16u;
     // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
     constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
-    int64_t i = 0;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
+    int64_t i = gid;                               // the CTA's i-th tile; group g takes i = g, g + NG, ...
+    for (int64_t tile = blockIdx.x + (int64_t)gid * gridDim.x; tile < ntiles; tile += (int64_t)NG * gridDim.x, i += NG) {
       const int s = (int)(i % STAGES);
       const uint32_t use = (uint32_t)(i / STAGES);
       const int64_t col = tile * T + c;
@@ -264,7 +277,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           g[n] = tp - B[(r0 + n) * T + c];
           tsum += tp;
         }
-        if (need_tsum) xsum[h][c] = tsum;          // the column mean needs the other half's sum too
+        if (need_tsum) xsum[gid][h][c] = tsum;          // the column mean needs the other half's sum too
         if constexpr (XM == 2) {                   // gossip Mix1 of this thread's rows, from the stage
           const int D1 = m1.D;                     // (uniform) -> a fully unrolled gather per slot count
           if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, xr);
@@ -277,9 +290,9 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }
-      named_bar_sync(1, CONS);                    // every consumer has read its theta_prev / theta_local
+      named_bar_sync(1 + 3 * gid, CONS);          // every consumer of the group has read its theta_prev / theta_local
       if (*(volatile int*)&abort_flag) break;     // uniform: the flag was written before the barrier
-      if (need_tsum) tsum += xsum[h ^ 1][c];
+      if (need_tsum) tsum += xsum[gid][h ^ 1][c];
       // ---- operands: g_hi over the theta_local box, g_lo over the theta_prev box
 #pragma unroll
       for (int n = 0; n < H; n += 4) {
@@ -294,8 +307,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      named_bar_sync(2, CONS);                    // operands complete; last tile's TMEM reads are done too
-      if (tid == 0) {
+      named_bar_sync(2 + 3 * gid, CONS);          // operands complete; last tile's TMEM reads are done too
+      if (lt == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_hi = smem_u32(B), a_lo = smem_u32(A);
         const uint32_t b_hi = smem_u32(wb_hi), b_lo = smem_u32(wb_lo);
@@ -307,7 +320,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           for (int ks = 0; ks < K / 8; ++ks) {
             const uint64_t da = umma_desc(aa + (uint32_t)ks * 256u, 128u, SBO, 0u);
             const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, SBO, 0u);
-            umma_tf32(tmem_base, da, db, idesc, (prod | ks) ? 1u : 0u);
+            umma_tf32(tmem_acc, da, db, idesc, (prod | ks) ? 1u : 0u);
           }
         }
         umma_commit(mma_bar);
@@ -325,7 +338,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         for (int m = 0; m < H; ++m) v[m] = vs;
       }
       if (need_tsum) xv = tsum * invK;
-      if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
+      if (!mbar_wait(mma_bar, (uint32_t)(i / NG) & 1)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }
@@ -335,7 +348,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
-      tmem_ld_cols<H>(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
+      tmem_ld_cols<H>(tmem_acc + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
       if constexpr (SUB) {
         if (!mix2_applies(a, col)) {
 #pragma unroll
@@ -361,9 +374,9 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         }
       }
       if (want_cd || a.x_next) {                   // column mean over both halves, then squared deviations
-        xchg[h][c] = asum;
-        named_bar_sync(3, CONS);
-        const float mean = (asum + xchg[h ^ 1][c]) * invK;
+        xchg[gid][h][c] = asum;
+        named_bar_sync(3 + 3 * gid, CONS);
+        const float mean = (asum + xchg[gid][h ^ 1][c]) * invK;
         if (a.x_next && live && h == 0) __stcs(a.x_next + col, mean);   // next round's global-average Mix1
         if (live && want_cd) {
 #pragma unroll
@@ -380,13 +393,13 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   // ---- wrap-up: tensor memory back, consensus partial sums (stage memory is free now)
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == CONS / 32) {
+  if (warp == ALLC / 32) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Shape::kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(NG * Shape::kTmemCols)) : "memory");
   }
   if (want_cd) {
-    double* red = reinterpret_cast<double*>(base);    // [CONS/32][H]: warps 0-3 hold workers 0-31, warps 4-7 workers 32-63
-    if (warp < CONS / 32) {
+    double* red = reinterpret_cast<double*>(base);    // [ALLC/32][H]; per group: warps 0-3 hold the first half of the workers, 4-7 the second
+    if (warp < ALLC / 32) {
 #pragma unroll
       for (int m = 0; m < H; ++m) {
         double d = (double)sacc[m];
@@ -400,7 +413,9 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       const int hh = tid / H, mm = tid % H;
       double d = 0.0;
 #pragma unroll
-      for (int w = 0; w < T / 32; ++w) d += red[(hh * (T / 32) + w) * H + mm];
+      for (int g = 0; g < NG; ++g)
+#pragma unroll
+        for (int w = 0; w < T / 32; ++w) d += red[((g * 2 + hh) * (T / 32) + w) * H + mm];
       a.partials[(size_t)blockIdx.x * KR + tid] = d;
     }
   }

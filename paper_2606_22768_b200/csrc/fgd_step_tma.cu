@@ -40,9 +40,10 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
   if (ta.n_tensors == 4)
     if (int rc = make_tensor_map(c, &tx, a.x, kTcCols, KP)) return rc;
   const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
-  auto launch = [&](auto kern) -> int {
-    if (int r = persistent_grid(c, kern, kTcConsumers + 32, Shape::kSmem, ntiles, grid)) return r;
-    kern<<<*grid, kTcConsumers + 32, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm, tx);
+  auto launch = [&](auto kern, int groups = 1) -> int {
+    const int block = groups * kTcConsumers + 32;
+    if (int r = persistent_grid(c, kern, block, Shape::kSmem, ntiles, grid)) return r;
+    kern<<<*grid, block, Shape::kSmem, st>>>(ta, d2, g1, tp, tl, tm, tx);
     return FGD_OK;
   };
   const bool full = c->K == KP;
@@ -53,7 +54,10 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
     default:
       if (a.n_ranges != 0)
         return full ? launch(outer_step_dense_tc_kernel<KP, 0, true, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false, true>);
-      return full ? launch(outer_step_dense_tc_kernel<KP, 0, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false>);
+      if constexpr (KP == 32)      // two consumer groups where the registers allow it
+        return full ? launch(outer_step_dense_tc_kernel<KP, 0, true, false, 2>, 2) : launch(outer_step_dense_tc_kernel<KP, 0, false, false, 2>, 2);
+      else
+        return full ? launch(outer_step_dense_tc_kernel<KP, 0, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false>);
   }
 }
 
