@@ -12,15 +12,6 @@
 
 using namespace fgd;
 
-namespace {
-
-int launch_finalize(fgd_ctx* c, int nblocks, double* out, cudaStream_t st) {
-  consensus_finalize_kernel<<<c->K, 32, 0, st>>>(c->partials, nblocks, c->K, out);
-  return check_launch(c, "consensus_finalize_kernel");
-}
-
-}  // namespace
-
 extern "C" {
 
 int fgd_create(fgd_ctx** out, int device, int K, int64_t P, int64_t ld) {
@@ -45,6 +36,8 @@ int fgd_create(fgd_ctx** out, int device, int K, int64_t P, int64_t ld) {
   if (e == cudaSuccess) e = cudaMalloc(&c->partials, sizeof(double) * (size_t)kMaxPartialBlocks * FGD_MAX_K);
   if (e == cudaSuccess) e = cudaMalloc(&c->status, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMalloc(&c->done, sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(c->done, 0, sizeof(unsigned int));
   if (e == cudaSuccess) {
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
@@ -66,6 +59,7 @@ int fgd_destroy(fgd_ctx* c) {
   DeviceGuard guard(c->device);
   cudaError_t e = cudaFree(c->partials);
   cudaFree(c->status);
+  cudaFree(c->done);
   delete c;
   return e == cudaSuccess ? FGD_OK : cuda_fail(nullptr, e, "fgd_destroy");
 }
@@ -250,6 +244,8 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   a.theta_new = theta_new;
   a.x = x;
   a.partials = cd_sumsq ? c->partials : nullptr;
+  a.cd_out = cd_sumsq;
+  a.done = c->done;
   a.P = c->P;
   a.ld = c->ld;
   a.K = K;
@@ -344,8 +340,7 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
     });
   }
   if (rc) return rc;
-  if (cd_sumsq) return launch_finalize(c, grid, cd_sumsq, st);
-  return FGD_OK;
+  return FGD_OK;   // (the consensus sums are finalised by the kernel's last CTA)
 }
 
 int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, void* stream) {
@@ -362,7 +357,7 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
   if ((K == 32 || K == 64) && pick_vec(4, c->P, c->ld, {theta}) == 4) {   // see consensus_split_kernel
     auto launch = [&](auto kern, int64_t ntiles) -> int {
       if (int r = persistent_grid(c, kern, kSplitBlock, 0, ntiles, &grid)) return r;
-      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld);
+      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld, cd_sumsq, c->done);
       return check_launch(c, "consensus_split_kernel");
     };
     const int64_t cols = 4 * kSplitBlock / (K / 16);           // columns per tile
@@ -370,18 +365,17 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
     if (int r = K == 64 ? launch(consensus_split_kernel<64, 4, 4, kSplitBlock>, ntiles)
                         : launch(consensus_split_kernel<32, 2, 4, kSplitBlock>, ntiles))
       return r;
-    return launch_finalize(c, grid, cd_sumsq, st);
+    return FGD_OK;
   }
   int rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
     const size_t smem = KTc > 0 ? 0 : sizeof(float) * (size_t)K * kBlock * (VECc + 1);
     auto kern = consensus_kernel<KTc, VECc, kBlock>;
     if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
-    kern<<<grid, kBlock, smem, st>>>(theta, c->partials, K, c->P, c->ld);
+    kern<<<grid, kBlock, smem, st>>>(theta, c->partials, K, c->P, c->ld, cd_sumsq, c->done);
     return check_launch(c, "consensus_kernel");
   });
-  if (rc) return rc;
-  return launch_finalize(c, grid, cd_sumsq, st);
+  return rc;
 }
 
 }  // extern "C"

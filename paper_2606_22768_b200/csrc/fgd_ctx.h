@@ -28,6 +28,7 @@ struct fgd_ctx {
   int64_t P = 0, ld = 0;
   int num_sms = 0;
   double* partials = nullptr;  // [kMaxPartialBlocks][K]
+  unsigned int* done = nullptr; // finished-CTA counter of the kernels that finalise the consensus sums themselves
   int* status = nullptr;       // device status word written by bounded waits that gave up
   int path = FGD_PATH_AUTO;    // which fused-step kernel family to use
   int max_smem_optin = 0;

@@ -41,6 +41,8 @@ struct StepArgs {
   float* theta_new;
   const float* x;       // XSRC_VECTOR: [P]; XSRC_MATRIX: [K, ld]; XSRC_FUSED: unused
   double* partials;     // [gridDim.x][K] consensus partial sums, or nullptr
+  double* cd_out;       // [K] consensus sums, written by the CTA that finishes last (with partials)
+  unsigned int* done;   // count of finished CTAs (zero between launches)
   int64_t P;
   int64_t ld;
   int K;

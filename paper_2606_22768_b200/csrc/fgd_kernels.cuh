@@ -219,6 +219,31 @@ __device__ __forceinline__ void block_reduce_partials(int K, AccFn acc, double* 
   }
 }
 
+// Second stage of the consensus sums, inside the producing kernel: every thread of every CTA calls
+// this after the CTA's row of partials[gridDim.x][K] is written.  The CTA that arrives last adds
+// the rows up -- one warp per worker, lanes stride the CTAs, then a shuffle tree: a fixed order,
+// so the result does not depend on which CTA happens to be last -- writes out[0..K) and re-arms
+// the counter for the next launch.  (out == nullptr: the caller reduces the partials itself.)
+__device__ __forceinline__ void finalize_in_last_cta(const double* partials, int K, double* out, unsigned int* counter) {
+  if (out == nullptr) return;
+  __shared__ int is_last;
+  __threadfence();                      // this CTA's partials are visible device-wide ...
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) + 1u == gridDim.x);   // ... before it is counted
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  for (int m = threadIdx.x >> 5; m < K; m += nwarps) {
+    double d = 0.0;
+    for (unsigned int b = lane; b < gridDim.x; b += 32) d += __ldcg(partials + (size_t)b * K + m);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) d += __shfl_down_sync(0xffffffffu, d, off);
+    if (lane == 0) out[m] = d;
+  }
+  if (threadIdx.x == 0) *counter = 0u;
+}
+
 // Same reduction for sums held in a register array (static indexing only).
 template <int BLOCK, int KR>
 __device__ __forceinline__ void block_reduce_regs(int K, const float (&sacc)[KR], double* partials) {
@@ -441,6 +466,7 @@ outer_step_kernel(const StepArgs a, const M2 m2, const GatherMix m1) {
     } else {
       block_reduce_partials<BLOCK>(K, [&](int m) { return sas[m * BLOCK + tid]; }, a.partials);
     }
+    finalize_in_last_cta(a.partials, K, a.cd_out, a.done);
   }
 }
 
@@ -545,7 +571,7 @@ outer_grad_kernel(const float* __restrict__ theta_prev, const float* __restrict_
 template <int KT, int VEC, int BLOCK>
 __global__ void __launch_bounds__(BLOCK)
 consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials, int Krt, int64_t P,
-                 int64_t ld) {
+                 int64_t ld, double* __restrict__ out, unsigned int* done) {
   extern __shared__ __align__(16) float smem[];
   const int K = KT > 0 ? KT : Krt;
   const int tid = threadIdx.x;
@@ -610,6 +636,7 @@ consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials,
   } else {
     block_reduce_partials<BLOCK>(K, [&](int m) { return sas[m * BLOCK + tid]; }, partials);
   }
+  finalize_in_last_cta(partials, K, out, done);
 }
 
 // Many workers (K = 32, 64): one thread per column would hold K values and K sums, which leaves one
@@ -619,7 +646,8 @@ consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials,
 // parity: one barrier per tile).
 template <int KT, int SPLIT, int VEC, int BLOCK>
 __global__ void __launch_bounds__(BLOCK)
-consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ partials, int64_t P, int64_t ld) {
+consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ partials, int64_t P, int64_t ld,
+                       double* __restrict__ out, unsigned int* done) {
   constexpr int R = KT / SPLIT;      // rows per thread
   constexpr int G = BLOCK / SPLIT;   // column groups per tile
   static_assert(KT % SPLIT == 0 && G % 32 == 0, "parts must be whole warps");
@@ -678,6 +706,7 @@ consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ par
     for (int w = 0; w < G / 32; ++w) d += red[q * (G / 32) + w][j];
     partials[(size_t)blockIdx.x * KT + tid] = d;
   }
+  finalize_in_last_cta(partials, KT, out, done);
 }
 
 // Global average with many workers, same split: out = column mean as one row (out_is_vector) or

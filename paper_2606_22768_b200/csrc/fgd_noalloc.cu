@@ -78,7 +78,7 @@ int launch_consensus(const float* theta, double* scratch, int K, int64_t P, int6
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return na_fail(FGD_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   }
-  kern<<<grid, kNoAllocBlock, smem, st>>>(theta, scratch, K, P, ld);
+  kern<<<grid, kNoAllocBlock, smem, st>>>(theta, scratch, K, P, ld, nullptr, nullptr);   // two-stage: finalised below
   return FGD_OK;
 }
 

@@ -418,6 +418,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         for (int w = 0; w < T / 32; ++w) d += red[((g * 2 + hh) * (T / 32) + w) * H + mm];
       a.partials[(size_t)blockIdx.x * KR + tid] = d;
     }
+    finalize_in_last_cta(a.partials, KR, a.cd_out, a.done);
   }
 }
 

@@ -388,6 +388,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
     for (int w = 0; w < NWARP; ++w) d += red[w][tid];
     a.partials[(size_t)blockIdx.x * K + tid] = d;
   }
+  if (want_cd) finalize_in_last_cta(a.partials, K, a.cd_out, a.done);
 }
 
 }  // namespace fgd
