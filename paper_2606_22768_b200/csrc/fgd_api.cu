@@ -296,7 +296,14 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   int grid = 0;
   int rc = FGD_OK;
   FgdTmaShape shape{0, 0, 0};
-  const bool can_tma = fgd_tma_eligible(c, a, dense2, &shape);
+  // Gather-heavy calls -- four or more neighbour slots in Mix2 together with a per-row x (a matrix,
+  // or a gossip Mix1 gathered in the kernel) -- wait on shared-memory loads with eight consumer warps
+  // (config 4: 88 % of the copy peak); sixteen warps of one column each hide that (96 %).  Every
+  // lighter call measured better with eight warps of two columns (config 3: 98 % vs 97 %; a ring
+  // Mix2 with a matrix-valued x: 93 % vs 92 %; a fused global average with four slots: 97 % vs 94 %).
+  const bool heavy = !dense2 && g2.kind == KMIX_GATHER && g2.D >= 4 &&
+                     (a.xsrc == XSRC_MATRIX || (a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER));
+  const bool can_tma = fgd_tma_eligible(c, a, dense2, heavy, &shape);
   // Worker counts up to 64 without a compile-time fp32 kernel of their own: the tensor-core kernel
   // is the fastest fused step we have there, and any mix is also a dense matrix -- so a gather /
   // mean Mix2 is densified and takes it too.

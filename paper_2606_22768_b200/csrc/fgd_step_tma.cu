@@ -112,9 +112,10 @@ int fgd_launch_mix_dense_tc(fgd_ctx* c, const float* in, float* out, const Dense
   return check_launch(c, "mix_dense_tc_kernel");
 }
 
-bool fgd_tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, FgdTmaShape* out) {
+bool fgd_tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, bool heavy, FgdTmaShape* out) {
   TmaShape sh{0, 0, 0};
-  if (!tma_eligible(c, a, dense2, &sh)) return false;
+  // `heavy` asks for the 512-consumer shape; worker counts without one fall back to the usual shapes
+  if (!(heavy && tma_eligible(c, a, dense2, true, &sh)) && !tma_eligible(c, a, dense2, false, &sh)) return false;
   out->vec = sh.vec;
   out->consumers = sh.consumers;
   out->stages = sh.stages;

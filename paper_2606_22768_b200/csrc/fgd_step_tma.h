@@ -11,7 +11,8 @@ struct FgdTmaShape {
   int vec, consumers, stages;
 };
 // Can the TMA kernel run this call?  Picks the tile shape.
-bool fgd_tma_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, FgdTmaShape* out);
+// heavy: the call gathers a lot per column (see fgd_outer_step_ex); such calls run with twice the consumer warps.
+bool fgd_tma_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, bool heavy, FgdTmaShape* out);
 int fgd_launch_step_tma(fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g2,
                         const fgd::DenseMix& d2, const fgd::GatherMix& g1, FgdTmaShape shape, cudaStream_t st,
                         int* grid_out);

@@ -64,7 +64,7 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   FGD_TMA_CASE(8, 4, 256) FGD_TMA_CASE(8, 4, 128)
   FGD_TMA_CASE(32, 1, 256) FGD_TMA_CASE(32, 1, 128)
 #elif FGD_TMA_GROUP == 2
-  FGD_TMA_CASE(16, 2, 256) FGD_TMA_CASE(16, 2, 128)
+  FGD_TMA_CASE(16, 2, 256) FGD_TMA_CASE(16, 2, 128) FGD_TMA_CASE(16, 1, 512)
   FGD_TMA_CASE(64, 1, 128)
 #endif
 #undef FGD_TMA_CASE

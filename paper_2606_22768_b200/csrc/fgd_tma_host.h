@@ -53,7 +53,7 @@ const int kTmaShapes[][3] = {  // {KT, vec, consumers}, in order of preference p
     {2, 4, 256}, {2, 4, 128},
     {4, 4, 256}, {4, 4, 128},
     {8, 4, 256}, {8, 4, 128},
-    {16, 2, 256}, {16, 2, 128},
+    {16, 1, 512}, {16, 2, 256}, {16, 2, 128},   // 512 x 1: gather-heavy calls (see fgd_tma_eligible)
     {32, 1, 256}, {32, 1, 128},
     {64, 1, 128},
 };
@@ -63,7 +63,7 @@ size_t tma_fixed_smem(int K, int KT, bool dense2, int consumers) {
 }
 
 // Can the TMA kernel run this call?  Picks the tile shape.
-bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* out) {
+bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, bool heavy, TmaShape* out) {
   if (!c->encode_tiled) return false;
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
@@ -72,6 +72,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, TmaShape* ou
   const size_t budget = (size_t)c->max_smem_optin - 6144;  // static shared memory (barriers, reduction buffer) + slack
   for (const auto& sh : kTmaShapes) {
     if (sh[0] != KT) continue;
+    if ((sh[2] == 512) != heavy) continue;   // 512 consumers: only, and always, for the gather-heavy calls
     const int vec = sh[1], consumers = sh[2];
     if (a.xsrc == XSRC_VECTOR && (reinterpret_cast<uintptr_t>(a.x) % (sizeof(float) * vec)) != 0) continue;
     if (a.x_next && (reinterpret_cast<uintptr_t>(a.x_next) % (sizeof(float) * vec)) != 0) continue;
