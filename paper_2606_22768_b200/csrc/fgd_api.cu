@@ -177,7 +177,8 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
       };
       int rc = FGD_OK;
       // compile-time worker counts also get a compile-time neighbour count (fully unrolled gathers)
-      const int dt = (KTc > 0 && gm.kind == KMIX_GATHER && (gm.D == 1 || gm.D == 2 || gm.D == 4)) ? gm.D : -1;
+      // (three slots run as four: unused slots carry weight 0 and point at the row itself)
+      const int dt = (KTc > 0 && gm.kind == KMIX_GATHER && gm.D >= 1 && gm.D <= 4) ? (gm.D == 3 ? 4 : gm.D) : -1;
       if constexpr (KTc > 0) {
         if (dt == 1) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 1>);
         else if (dt == 2) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 2>);
@@ -307,7 +308,12 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   // Worker counts up to 64 without a compile-time fp32 kernel of their own: the tensor-core kernel
   // is the fastest fused step we have there, and any mix is also a dense matrix -- so a gather /
   // mean Mix2 is densified and takes it too.
-  bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, dense2, g1);
+  // K = 32 has a compile-time fp32 kernel that is the faster one for a light sparse Mix2 (at most two
+  // neighbour slots) with x one value per column or gathered in the kernel (ring: 5.8 / 5.1 TB/s
+  // against 5.6 / 4.9); with more slots (hypercube: 2.4 TB/s against 5.6) or a matrix-valued x
+  // (5.1 against 5.8) the tensor-core kernel wins.
+  const bool tc_at_32 = dense2 || (g2.kind == KMIX_GATHER && g2.D > 2) || a.xsrc == XSRC_MATRIX;
+  bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, tc_at_32, g1);
   if (can_tc && !dense2) {
     double Wd[FGD_MAX_K * FGD_MAX_K];
     if (fgd_dense_matrix(mix2, Wd) != FGD_OK) can_tc = false;

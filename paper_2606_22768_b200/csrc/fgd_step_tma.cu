@@ -14,11 +14,12 @@ int fgd_launch_step_tma_g2(fgd_ctx*, const StepArgs&, bool, const GatherMix&, co
 
 // Tensor-core dense step: Mix1 given (row or matrix) or fused (mean or gossip); K = 64 and every worker
 // count in [17, 63] that has no compile-time fp32 kernel of its own (zero-padded to 32, 48 or 64),
-// plus K = 32 when Mix2 really is dense (`really_dense`: the caller's matrix, not a densified gather).
-bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool really_dense, const GatherMix& g1) {
+// plus K = 32 when the caller says so (`tc_at_32`: a dense Mix2, or a sparse one the fp32 kernel
+// is slow on).
+bool fgd_tc_eligible(const fgd_ctx* c, const StepArgs& a, bool tc_at_32, const GatherMix& g1) {
   const int K = c->K;
   if (K > kTcMaxK || K < kTcMinK) return false;
-  if (kt_of(K) == 16 || (kt_of(K) == 32 && !really_dense)) return false;
+  if (kt_of(K) == 16 || (kt_of(K) == 32 && !tc_at_32)) return false;
   if (!c->encode_tiled) return false;
   // column-range Mix2 is built for the one-value-per-column Mix1 (the "-subset" configurations pair it
   // with the global average)

@@ -17,7 +17,7 @@ int fgd_launch_step_tma(fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const f
                         const fgd::DenseMix& d2, const fgd::GatherMix& g1, FgdTmaShape shape, cudaStream_t st,
                         int* grid_out);
 // Dense Mix2 on the tensor cores (17 <= K <= 64, padded to 32 / 48 / 64 workers).
-bool fgd_tc_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool really_dense, const fgd::GatherMix& g1);
+bool fgd_tc_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool tc_at_32, const fgd::GatherMix& g1);
 // Stand-alone mix on the tensor cores (dm holds the dense, transposed matrix of whatever mix it is).
 bool fgd_mix_tc_eligible(const fgd_ctx* c, const float* in, bool really_dense);
 int fgd_launch_mix_dense_tc(fgd_ctx* c, const float* in, float* out, const fgd::DenseMix& dm, cudaStream_t st);

@@ -25,10 +25,11 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   // neighbour count of a gather Mix2 as a template argument when it is one of the common ones
   // (identity 0, one-peer / matching 1, ring 2, hypercube of 16 workers 4); else read at run time
   int d2t = -1;
-  if (!dense2 && g2.kind == KMIX_GATHER && (g2.D == 0 || g2.D == 1 || g2.D == 2 || g2.D == 4)) d2t = g2.D;
+  // (three slots run as four: unused slots carry weight 0 and point at the row itself)
+  if (!dense2 && g2.kind == KMIX_GATHER && g2.D <= 4) d2t = g2.D == 3 ? 4 : g2.D;
   // a fused gather Mix1 with the same neighbour count as Mix2 (both mixes on one topology, as in
   // the paper's LocalM1M2) also gets a static gather
-  const bool same_d1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER && d2t > 0 && g1.D == d2t;
+  const bool same_d1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER && d2t > 0 && (g1.D == d2t || (g1.D == 3 && d2t == 4));
   auto go = [&]<int KTc, int VECc, int Cc, int D2c, bool SAME1>() -> int {
     int grid = 0;
     if constexpr (D2c == -2) {

@@ -57,7 +57,7 @@ MIX_CASES = [
     # tensor-core mix: worker counts 17..64 (zero-padded to 32 / 48 / 64), sparse mixes densified
     (48, 9001, ("ring",)), (40, 5000, ("dense", gen.sinkhorn_W(8, 40))), (33, 4100, ("matching",)), (63, 3000, ("mean",)),
     (32, 6002, ("dense", gen.sinkhorn_W(7, 32))), (24, 7000, ("ring", 0.3)), (17, 2000, ("dense", gen.sinkhorn_W(9, 17))),
-    (64, 20000, ("hypercube", 0.1)), (16, 9000, ("randgraph", 5, 0.2)), (40, 3000, ("randgraph", 3)), (7, 2000, ("randgraph", 2)),
+    (64, 20000, ("hypercube", 0.1)), (8, 30000, ("hypercube", 0.2)), (16, 9000, ("randgraph", 5, 0.2)), (40, 3000, ("randgraph", 3)), (7, 2000, ("randgraph", 2)),
 ]
 
 
@@ -155,6 +155,11 @@ STEP_CASES = [
     (64, 3000, ("identity",), ("ring",)),
     (32, 6000, ("matching",), ("dense", gen.sinkhorn_W(7, 32))),
     (56, 3001, ("circulant", 4, 0.2), ("circulant", 3)),
+    # three neighbour slots run as the compile-time four; five at K = 32 go to the tensor-core kernel
+    (8, 9000, ("hypercube", 0.2), ("hypercube",)),
+    (8, 5001, ("mean",), ("hypercube", 0.3)),
+    (32, 7000, ("hypercube",), ("hypercube", 0.1)),
+    (32, 4001, ("mean",), ("hypercube",)),
     # fewer columns than one tile (and than one vector)
     (64, 5, ("mean",), ("dense", SINK64)),
     (48, 1, ("mean",), ("ring",)),
