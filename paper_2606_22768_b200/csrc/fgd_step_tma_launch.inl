@@ -25,11 +25,16 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   // neighbour count of a gather Mix2 as a template argument when it is one of the common ones
   // (identity 0, one-peer / matching 1, ring 2, hypercube of 16 workers 4); else read at run time
   int d2t = -1;
-  // (three slots run as four: unused slots carry weight 0 and point at the row itself)
-  if (!dense2 && g2.kind == KMIX_GATHER && g2.D <= 4) d2t = g2.D == 3 ? 4 : g2.D;
+  // (three slots run as four, five to seven as eight: unused slots carry weight 0 and point at the
+  // row itself; the eight-slot kernels exist for K = 8 and 16)
+  if (!dense2 && g2.kind == KMIX_GATHER) {
+    if (g2.D <= 4) d2t = g2.D == 3 ? 4 : g2.D;
+    else if (KT == 8 || KT == 16) d2t = 8;
+  }
   // a fused gather Mix1 with the same neighbour count as Mix2 (both mixes on one topology, as in
   // the paper's LocalM1M2) also gets a static gather
-  const bool same_d1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER && d2t > 0 && (g1.D == d2t || (g1.D == 3 && d2t == 4));
+  const bool same_d1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER && d2t > 0 &&
+                       (g1.D == d2t || (g1.D == 3 && d2t == 4) || (g1.D > 4 && d2t == 8));
   auto go = [&]<int KTc, int VECc, int Cc, int D2c, bool SAME1>() -> int {
     int grid = 0;
     if constexpr (D2c == -2) {
@@ -57,17 +62,22 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
       default: return go.template operator()<kt, v, cc, -1, false>();                       \
     }                                                                                       \
   }
+// the same plus the eight-slot kernels
+#define FGD_TMA_CASE8(kt, v, cc)                                                            \
+  if (KT == kt && sh.vec == v && sh.consumers == cc && !dense2 && d2t == 8) { FGD_TMA_D(kt, v, cc, 8) }  \
+  FGD_TMA_CASE(kt, v, cc)
 #if FGD_TMA_GROUP == 0
   FGD_TMA_CASE(0, 2, 256) FGD_TMA_CASE(0, 1, 256) FGD_TMA_CASE(0, 1, 128)
   FGD_TMA_CASE(2, 4, 256) FGD_TMA_CASE(2, 4, 128)
   FGD_TMA_CASE(4, 4, 256) FGD_TMA_CASE(4, 4, 128)
 #elif FGD_TMA_GROUP == 1
-  FGD_TMA_CASE(8, 4, 256) FGD_TMA_CASE(8, 4, 128)
+  FGD_TMA_CASE8(8, 4, 256) FGD_TMA_CASE8(8, 4, 128)
   FGD_TMA_CASE(32, 1, 256) FGD_TMA_CASE(32, 1, 128)
 #elif FGD_TMA_GROUP == 2
-  FGD_TMA_CASE(16, 2, 256) FGD_TMA_CASE(16, 2, 128) FGD_TMA_CASE(16, 1, 512)
+  FGD_TMA_CASE8(16, 2, 256) FGD_TMA_CASE8(16, 2, 128) FGD_TMA_CASE8(16, 1, 512)
   FGD_TMA_CASE(64, 1, 128)
 #endif
+#undef FGD_TMA_CASE8
 #undef FGD_TMA_CASE
 #undef FGD_TMA_D
   return fail(c, FGD_ERR_UNSUPPORTED, "internal: no TMA kernel for this shape");
