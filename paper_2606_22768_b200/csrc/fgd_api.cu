@@ -177,12 +177,16 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
       };
       int rc = FGD_OK;
       // compile-time worker counts also get a compile-time neighbour count (fully unrolled gathers)
-      // (three slots run as four: unused slots carry weight 0 and point at the row itself)
-      const int dt = (KTc > 0 && gm.kind == KMIX_GATHER && gm.D >= 1 && gm.D <= 4) ? (gm.D == 3 ? 4 : gm.D) : -1;
+      // (three slots run as four, five to seven as eight -- K = 8 and 16 only: unused slots carry
+      // weight 0 and point at the row itself)
+      int dt = -1;
+      if (KTc > 0 && gm.kind == KMIX_GATHER && gm.D >= 1)
+        dt = gm.D <= 4 ? (gm.D == 3 ? 4 : gm.D) : ((KTc == 8 || KTc == 16) ? 8 : -1);
       if constexpr (KTc > 0) {
         if (dt == 1) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 1>);
         else if (dt == 2) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 2>);
         else if (dt == 4) rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix, 4>);
+        else if (dt == 8) rc = launch(mix_kernel<(KTc == 8 || KTc == 16) ? KTc : 8, VECc, false, kBlock, GatherMix, 8>);
         else rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix>);
       } else {
         rc = launch(mix_kernel<KTc, VECc, false, kBlock, GatherMix>);
