@@ -76,6 +76,8 @@ def parse_args():
                     help="variant: Mix1 computed inside the fused step from the staged theta_prev (one launch per round, 20 B per worker-parameter)")
     ap.add_argument("--graph", action="store_true",
                     help="variant: capture the round (Mix1 + fused step) into one CUDA graph and time its replays")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the round: the fused step across worker counts and mix kinds (4 GB per tensor)")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
@@ -254,6 +256,10 @@ def run_ours(args):
     if args.js:
         if rank == 0:
             print(json.dumps(js_table(torch, fgd, dev, measured_peak())), flush=True)
+        return
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak())), flush=True)
         return
     cfg = dict(CONFIGS[args.config])
     if args.cols:
@@ -451,6 +457,45 @@ def kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, peak, r
         gbs = nbytes / (ms * 1e-3) / 1e9
         out["kernels"][name] = {"ms": round(ms, 4), "algorithmic_gb": round(nbytes / 1e9, 2), "gbs": round(gbs, 1),
                                 "frac": round(gbs / peak[0], 3)}
+    return out
+
+
+def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
+                Ks=(2, 3, 4, 6, 8, 12, 16, 17, 24, 32, 40, 48, 56, 63, 64)):
+    """Fused outer step (in place, consensus sums on) across worker counts at a fixed tensor size:
+    Mix2 = ring / hypercube (powers of two) / dense Sinkhorn with x one value per column, and the
+    fully fused ring-ring round.  GB/s = algorithmic bytes (20 K P + 4 P, or 20 K P fused) / time."""
+    out = {"peak_gbs": peak[0], "peak_kind": peak[1], "tensor_bytes": tensor_bytes, "unit": "GB/s", "rows": {}}
+    for K in Ks:
+        P = tensor_bytes // 4 // K // 128 * 128
+        tp = torch.empty((K, P), dtype=torch.float32, device=dev).normal_(0.0, 0.02)
+        tl = tp + 1e-3 * torch.randn_like(tp)
+        v = torch.zeros_like(tp)
+        x = tp.mean(0).contiguous()
+        cd = torch.zeros(K, dtype=torch.float64, device=dev)
+        ctx = fgd.Context(K, P, device=dev.index or 0)
+        ring = fgd.MixDesc.ring(K)
+        cases = {"ring": (ring, None), "dense": (fgd.MixDesc.dense(gen.sinkhorn_W(0, K)), None), "ring+ring fused": (ring, ring)}
+        if K & (K - 1) == 0 and K > 1:
+            cases["hypercube"] = (fgd.MixDesc.hypercube(K), None)
+        row = {}
+        for name, (m2, m1) in cases.items():
+            f = ((lambda: fgd.fgd_outer_step(ctx, m2, m1, None, False, tl, tp, v, tp, 0.7, 0.9, cd)) if m1 is not None
+                 else (lambda: fgd.fgd_outer_step(ctx, m2, None, x, True, tl, tp, v, tp, 0.7, 0.9, cd)))
+            for _ in range(3):
+                f()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                f()
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            nbytes = 20 * K * P + (0 if m1 is not None else 4 * P)
+            row[name] = round(nbytes / (ms * 1e-3) / 1e9)
+        out["rows"][str(K)] = row
+        del tp, tl, v, x
     return out
 
 

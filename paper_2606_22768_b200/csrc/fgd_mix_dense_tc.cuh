@@ -166,8 +166,7 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
         float* const out_col = a.out + (size_t)r0 * ld + col;
 #pragma unroll
         for (int m = 0; m < H; ++m) {
-          if (!FULL && m >= hr) break;
-          __stcs(out_col + (size_t)m * ld, r[m]);
+          if (FULL || m < hr) __stcs(out_col + (size_t)m * ld, r[m]);
         }
       }
     }

@@ -133,6 +133,8 @@ __device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A,
 // registers each: that fits the 32-worker shape (measured: K = 17 3.3 -> 4.7 TB/s, K = 24 4.6 ->
 // 5.7, dense K = 32 5.4 -> 5.6) and spills at 48 and 64 workers (K = 64: 10.8 -> 13.8 ms), which
 // therefore keep one group.
+// (registers are handed out per four warps: 288 threads count as 384, i.e. at most 168 registers
+// each, and 544 as 640, i.e. 96 -- asking for more makes the kernel unlaunchable)
 template <int KP, int XM, bool FULL, bool SUB = false, int NG = 1>
 __global__ void __launch_bounds__(NG * kTcConsumers + 32)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
@@ -258,8 +260,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       if constexpr (XM == 1) {                     // now so that they arrive behind the TMA wait and the MMA
         if (live) {
 #pragma unroll
-          for (int m = 0; m < H; ++m)
-            if (FULL || m < hr) xr[m] = __ldcs(a.x + (size_t)(r0 + m) * ld + col);
+          for (int m = 0; m < H; ++m) xr[m] = (FULL || m < hr) ? __ldcs(a.x + (size_t)(r0 + m) * ld + col) : 0.f;
         }
       }
       unsigned char* stage = base + (size_t)s * 3 * kTcBox;
@@ -362,15 +363,24 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         float* const new_col = a.theta_new + (size_t)r0 * ld + col;
 #pragma unroll
         for (int m = 0; m < H; ++m) {
-          if (!FULL && m >= hr) break;
+          // With a per-row x the padded rows are computed like the others (their inputs are zeros)
+          // and only kept out of the stores and of the column sum: an early exit from the unrolled
+          // loop cost those register-heavy variants half their speed.  Without one it is the
+          // faster form.
+          if constexpr (!XMAT) {
+            if (!FULL && m >= hr) break;
+          }
+          const bool row_live = FULL || m < hr;
           const float vn = fmaf(mu, v[m], gh[m]);
           float xm = xv;
           if constexpr (XMAT) xm = xr[m];
           const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xm);
-          __stcs(mom_col + (size_t)m * ld, vn);
-          __stcs(new_col + (size_t)m * ld, tn);
+          if (row_live) {
+            __stcs(mom_col + (size_t)m * ld, vn);
+            __stcs(new_col + (size_t)m * ld, tn);
+          }
           v[m] = tn;
-          asum += tn;
+          asum += row_live ? tn : 0.f;
         }
       }
       if (want_cd || a.x_next) {                   // column mean over both halves, then squared deviations
@@ -380,8 +390,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         if (a.x_next && live && h == 0) __stcs(a.x_next + col, mean);   // next round's global-average Mix1
         if (live && want_cd) {
 #pragma unroll
-          for (int m = 0; m < H; ++m) {
-            if (!FULL && m >= hr) break;
+          for (int m = 0; m < H; ++m) {            // (sums of padded rows are never read)
             const float d = v[m] - mean;
             sacc[m] = fmaf(d, d, sacc[m]);
           }
