@@ -177,6 +177,9 @@ int kt_of(int K) {
     default: return 0;
   }
 }
+// The TMA-pipelined fused step is also instantiated for 3, 6 and 12 workers (clusters that are not
+// a power of two); the stand-alone kernels and the register path run those with run-time K.
+int kt_tma_of(int K) { return (K == 3 || K == 6 || K == 12) ? K : kt_of(K); }
 int want_vec(int KT) { return KT == 0 ? 1 : (KT <= 16 ? 4 : (KT == 32 ? 2 : 1)); }
 
 // Calls f.template operator()<KT, VEC>() for the (KT, VEC) pair chosen at run time.

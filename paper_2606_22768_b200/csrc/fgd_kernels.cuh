@@ -271,7 +271,7 @@ __device__ __forceinline__ void block_reduce_regs(int K, const float (&sacc)[KR]
 // the MB weights of a step are one or two 128-bit broadcast reads.  fn(m, out_m) consumes a row.
 template <int KT, int VEC, int BLOCK, bool FULL_UNROLL, typename RowFn>
 __device__ __forceinline__ void dense_rows(int K, const float* wts, const float* cols, int tid, RowFn fn) {
-  constexpr int MB = (KT > 0 && KT < 8) ? KT : 8;
+  constexpr int MB = (KT > 0 && KT < 8) ? KT : ((KT > 0 && KT % 8 != 0) ? 4 : 8);   // MB divides a compile-time K
   constexpr bool VECW = (KT > 0) && (KT % 4 == 0);   // rows of Wt are 16-byte aligned
 #pragma unroll(FULL_UNROLL ? 8 : 1)
   for (int mb = 0; mb < K; mb += MB) {

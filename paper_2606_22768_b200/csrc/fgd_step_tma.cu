@@ -11,6 +11,7 @@ using namespace fgd;
 int fgd_launch_step_tma_g0(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 int fgd_launch_step_tma_g1(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 int fgd_launch_step_tma_g2(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
+int fgd_launch_step_tma_g3(fgd_ctx*, const StepArgs&, bool, const GatherMix&, const DenseMix&, const GatherMix&, FgdTmaShape, cudaStream_t, int*);
 
 // Tensor-core dense step: Mix1 given (row or matrix) or fused (mean or gossip); K = 64 and every worker
 // count in [17, 63] that has no compile-time fp32 kernel of its own (zero-padded to 32, 48 or 64),
@@ -125,7 +126,8 @@ bool fgd_tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, bool hea
 
 int fgd_launch_step_tma(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
                         const GatherMix& g1, FgdTmaShape shape, cudaStream_t st, int* grid_out) {
-  switch (kt_of(c->K)) {
+  switch (kt_tma_of(c->K)) {
+    case 3: case 6: case 12: return fgd_launch_step_tma_g3(c, a, dense2, g2, d2, g1, shape, st, grid_out);
     case 0: case 2: case 4: return fgd_launch_step_tma_g0(c, a, dense2, g2, d2, g1, shape, st, grid_out);
     case 8: case 32: return fgd_launch_step_tma_g1(c, a, dense2, g2, d2, g1, shape, st, grid_out);
     default: return fgd_launch_step_tma_g2(c, a, dense2, g2, d2, g1, shape, st, grid_out);

@@ -7,7 +7,7 @@ using namespace fgd;
 namespace {
 static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
                     const GatherMix& g1, TmaShape sh, cudaStream_t st, int* grid_out) {
-  const int K = c->K, KT = kt_of(K);
+  const int K = c->K, KT = kt_tma_of(K);
   TmaStepArgs ta;
   ta.s = a;
   ta.status = c->status;
@@ -26,10 +26,10 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   // (identity 0, one-peer / matching 1, ring 2, hypercube of 16 workers 4); else read at run time
   int d2t = -1;
   // (three slots run as four, five to seven as eight: unused slots carry weight 0 and point at the
-  // row itself; the eight-slot kernels exist for K = 8 and 16)
+  // row itself; the eight-slot kernels exist for K = 8, 12 and 16)
   if (!dense2 && g2.kind == KMIX_GATHER) {
     if (g2.D <= 4) d2t = g2.D == 3 ? 4 : g2.D;
-    else if (KT == 8 || KT == 16) d2t = 8;
+    else if (KT == 8 || KT == 12 || KT == 16) d2t = 8;
   }
   // a fused gather Mix1 with the same neighbour count as Mix2 (both mixes on one topology, as in
   // the paper's LocalM1M2) also gets a static gather
@@ -76,6 +76,10 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
 #elif FGD_TMA_GROUP == 2
   FGD_TMA_CASE8(16, 2, 256) FGD_TMA_CASE8(16, 2, 128) FGD_TMA_CASE8(16, 1, 512)
   FGD_TMA_CASE(64, 1, 128)
+#elif FGD_TMA_GROUP == 3
+  FGD_TMA_CASE(3, 4, 256) FGD_TMA_CASE(3, 4, 128)
+  FGD_TMA_CASE(6, 4, 256) FGD_TMA_CASE(6, 4, 128)
+  FGD_TMA_CASE8(12, 2, 256) FGD_TMA_CASE8(12, 2, 128)
 #endif
 #undef FGD_TMA_CASE8
 #undef FGD_TMA_CASE

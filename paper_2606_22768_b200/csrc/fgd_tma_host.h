@@ -51,8 +51,11 @@ struct TmaShape {
 const int kTmaShapes[][3] = {  // {KT, vec, consumers}, in order of preference per KT
     {0, 2, 256}, {0, 1, 256}, {0, 1, 128},   // run-time K: widest tile whose two stages fit
     {2, 4, 256}, {2, 4, 128},
+    {3, 4, 256}, {3, 4, 128},
     {4, 4, 256}, {4, 4, 128},
+    {6, 4, 256}, {6, 4, 128},
     {8, 4, 256}, {8, 4, 128},
+    {12, 2, 256}, {12, 2, 128},
     {16, 1, 512}, {16, 2, 256}, {16, 2, 128},   // 512 x 1: gather-heavy calls (see fgd_tma_eligible)
     {32, 1, 256}, {32, 1, 128},
     {64, 1, 128},
@@ -68,7 +71,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, bool heavy, 
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
-  const int K = c->K, KT = kt_of(K), NT = tma_n_tensors(a, KT, dense2);
+  const int K = c->K, KT = kt_tma_of(K), NT = tma_n_tensors(a, KT, dense2);
   const size_t budget = (size_t)c->max_smem_optin - 6144;  // static shared memory (barriers, reduction buffer) + slack
   for (const auto& sh : kTmaShapes) {
     if (sh[0] != KT) continue;
