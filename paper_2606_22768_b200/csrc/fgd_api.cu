@@ -330,10 +330,10 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   if (can_tc && c->path != FGD_PATH_REGISTER) {
     rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
-  } else if (can_tma && c->path != FGD_PATH_REGISTER && !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && KT == 16)))) {
+  } else if (can_tma && c->path != FGD_PATH_REGISTER && !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && (KT == 8 || KT == 16))))) {
     // (AUTO keeps the register kernel with one or two workers, where a tile is too little work per
-    // pipeline hand-off, and for a dense Mix2 at K = 16, where its all-register W g product measured
-    // 6.1 TB/s against 5.0 TB/s for the shared-memory version of the pipelined kernel)
+    // pipeline hand-off, and for a dense Mix2 at K = 8 and 16, where its all-register W g product
+    // measured 5.9 / 6.1 TB/s against 5.2 / 5.0 TB/s for the shared-memory version of the pipelined kernel)
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next});
