@@ -5,23 +5,29 @@
 // about a quarter of the HBM roofline).  Here it runs as tcgen05.mma.kind::tf32 with the
 // error-compensated three-product split
 //     W g  ~=  W_hi g_hi + W_hi g_lo + W_lo g_hi          (hi = tf32-rounded, lo = remainder)
-// accumulated in fp32 in tensor memory, which keeps the result within fp32 rounding of the
-// exact product (a single tf32 product would miss the 1e-5 parity bar).
+// accumulated in fp32 in tensor memory: relative error about 2^-22 of sum |W||g| (the remainders
+// are themselves cut to tf32 and the lo x lo term is dropped) -- four times fp32 rounding, well
+// inside the 1e-5 parity bar that a single tf32 product would miss.
 //
 // Mapping.  The 128 columns of a tile are the M dimension of the MMA, the K workers n are its
 // K dimension and the K output rows m its N dimension:
 //     D[col][m] += A[col][n] * B[n][m],   A = g^T, B = W^T, both K-major (worker-contiguous).
-// D row `col` lives in TMEM lane `col`, so after tcgen05.ld thread `col` holds ghat[0..K-1] of
-// ITS column in registers -- the same thread-owns-a-column layout as the other kernels; the
-// Nesterov update, the streaming stores and the consensus sums follow without any exchange.
+// D row `col` lives in TMEM lane `col`, so after tcgen05.ld the two threads of column `col` hold
+// its ghat values in registers -- the same thread-owns-a-column layout as the other kernels;
+// the Nesterov update, the streaming stores and the consensus sums follow with one exchange of
+// the column sum.
 //
 // Pipeline per CTA (one per SM): a producer warp streams [K x 128] boxes of theta_prev,
-// theta_local and momentum into a shared-memory ring (2 stages at K = 64, 4 at K = 32) with 2-D
-// TMA loads; the eight consumer warps (two threads per column, half of the workers each) compute g = theta_prev - theta_local in registers, split it and write g_hi /
-// g_lo IN PLACE over the theta_local / theta_prev boxes of the stage in the K-major core-matrix
-// operand layout (a thread's four consecutive workers are one 16-byte row of a core matrix, so
-// its stores are 128-bit and conflict-free); one thread issues the 3 x (K/8) MMAs and commits them to an
-// mbarrier; every consumer then reads its accumulator row from TMEM.
+// theta_local and momentum into a shared-memory ring (2 stages at K = 64 and 48, 4 at K = 32)
+// with 2-D TMA loads; the eight consumer warps (two threads per column, half of the workers
+// each) compute g = theta_prev - theta_local in registers, split it and write g_hi / g_lo IN
+// PLACE over the theta_local / theta_prev boxes of the stage in the K-major core-matrix operand
+// layout (a thread's four consecutive workers are one 16-byte row of a core matrix, so its
+// stores are 128-bit and conflict-free); one thread issues the 3 x (K/8) MMAs and commits them
+// to an mbarrier; every consumer then reads its accumulator row from TMEM.
+// Worker counts between the shapes are zero-padded (FULL), Mix1 may be given, a fused mean or a
+// fused sparse mix (XM), Mix2 may be restricted to column ranges (SUB), and the 32-worker shape
+// runs two consumer groups (NG): see the template parameters below.
 // All waits are bounded; tensor memory is always released before the kernel returns.
 #ifndef FGD_STEP_DENSE_TC_CUH_
 #define FGD_STEP_DENSE_TC_CUH_
