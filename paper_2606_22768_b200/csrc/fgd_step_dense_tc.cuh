@@ -104,22 +104,41 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&r)[N]) {
   tmem_ld_wait();
 }
 
+// 32 lanes x 32 bit x 8 columns, registers -> tensor memory (this thread's lane); tmem_st_wait()
+// orders the stores before later tensor-memory reads of the same thread.
+__device__ __forceinline__ void tmem_st_8(uint32_t taddr, const float* r) {
+  const uint32_t* u = reinterpret_cast<const uint32_t*>(r);
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // Sparse Mix1 of the rows [r0, r0 + H) of one column from a staged [K][T] box of theta_prev.
 // DJ >= the used slot count: unused slots point at the row itself with weight 0, padded rows have
 // all-zero weights, so neither needs a branch; all loads of a row are issued before its FMAs.
 template <int DJ, int H, int T>
-__device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A, int r0, int c, float (&xr)[H]) {
+// The H results go to this thread's tensor-memory scratch columns [tx, tx + H), eight at a time:
+// they are needed again only in the epilogue, and with all shared memory given to the stages a
+// spilled register goes all the way to L2.
+__device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A, int r0, int c, uint32_t tx) {
 #pragma unroll
-  for (int m = 0; m < H; ++m) {
-    const int r = r0 + m;
-    float t[DJ > 0 ? DJ : 1];
+  for (int mb = 0; mb < H; mb += 8) {
+    float x8[8];
 #pragma unroll
-    for (int j = 0; j < DJ; ++j) t[j] = A[m1.nbr[r * FGD_MAX_D + j] * T + c];
-    float acc = m1.w_self[r] * A[r * T + c];
+    for (int q = 0; q < 8; ++q) {
+      const int r = r0 + mb + q;
+      float t[DJ > 0 ? DJ : 1];
 #pragma unroll
-    for (int j = 0; j < DJ; ++j) acc = fmaf(m1.w[r * FGD_MAX_D + j], t[j], acc);
-    xr[m] = acc;
+      for (int j = 0; j < DJ; ++j) t[j] = A[m1.nbr[r * FGD_MAX_D + j] * T + c];
+      float acc = m1.w_self[r] * A[r * T + c];
+#pragma unroll
+      for (int j = 0; j < DJ; ++j) acc = fmaf(m1.w[r * FGD_MAX_D + j], t[j], acc);
+      x8[q] = acc;
+    }
+    tmem_st_8(tx + (uint32_t)mb, x8);
   }
+  tmem_st_wait();
 }
 
 // XM: where the Mix1 result x comes from.  0 = one value per column (a given row, or the column
@@ -151,6 +170,10 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
   constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
   constexpr int ALLC = NG * CONS;                   // all consumer threads; the producer warp follows them
+  // tensor memory: the accumulator columns of every group, then (fused sparse Mix1) as many scratch
+  // columns for x; 32 + 32, 64 + 64: powers of two
+  constexpr int kTmemAll = NG * Shape::kTmemCols + (XM == 2 ? Shape::kTmemCols : 0);
+  static_assert(XM != 2 || NG == 1, "the x scratch columns are laid out for one consumer group");
   static_assert(STAGES % NG == 0, "every stage belongs to one group");
   const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -194,7 +217,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     *reinterpret_cast<float*>(wb_lo + off) = w - hi;
   }
   if (warp == ALLC / 32) {   // the producer warp owns tensor memory: allocate the accumulator columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(NG * Shape::kTmemCols)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)kTmemAll) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // W operands are read by the MMA (async proxy)
@@ -244,6 +267,9 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     // TMEM and barrier latencies, and half-length arrays keep everything in registers.
     const int lt = tid & (CONS - 1);              // index within the group
     const int c = lt & (T - 1), h = lt >> 7, r0 = h * H;
+    const uint32_t tmem_lane = (uint32_t)((warp & 3) * 32) << 16;      // this warp's quarter of the lanes
+    // scratch columns of this thread for a fused sparse Mix1 result (behind all accumulator columns)
+    const uint32_t tmem_x = tmem_base + (uint32_t)(NG * Shape::kTmemCols) + tmem_lane + (uint32_t)r0;
     const float invK = 1.0f / (float)KR;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
     const float lr = a.lr, mu = a.mu;
@@ -262,7 +288,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       const bool live = col < P;
       float xv = 0.f;
       if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
-      float xr[XMAT ? H : 1];                      // a matrix-valued Mix1 result: this thread's rows, requested
+      float xr[XM == 1 ? H : 1];                   // a matrix-valued Mix1 result: this thread's rows, requested
       if constexpr (XM == 1) {                     // now so that they arrive behind the TMA wait and the MMA
         if (live) {
 #pragma unroll
@@ -287,11 +313,11 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         if (need_tsum) xsum[gid][h][c] = tsum;          // the column mean needs the other half's sum too
         if constexpr (XM == 2) {                   // gossip Mix1 of this thread's rows, from the stage
           const int D1 = m1.D;                     // (uniform) -> a fully unrolled gather per slot count
-          if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, xr);
-          else if (D1 == 1) tc_gather_x<1, H, T>(m1, A, r0, c, xr);
-          else if (D1 == 2) tc_gather_x<2, H, T>(m1, A, r0, c, xr);
-          else if (D1 <= 4) tc_gather_x<4, H, T>(m1, A, r0, c, xr);
-          else tc_gather_x<FGD_MAX_D, H, T>(m1, A, r0, c, xr);
+          if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, tmem_x);
+          else if (D1 == 1) tc_gather_x<1, H, T>(m1, A, r0, c, tmem_x);
+          else if (D1 == 2) tc_gather_x<2, H, T>(m1, A, r0, c, tmem_x);
+          else if (D1 <= 4) tc_gather_x<4, H, T>(m1, A, r0, c, tmem_x);
+          else tc_gather_x<FGD_MAX_D, H, T>(m1, A, r0, c, tmem_x);
         }
       } else {
         *(volatile int*)&abort_flag = 1;
@@ -354,8 +380,41 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float asum = 0.f;
+      if constexpr (XM == 2) {
+        // ---- phase 2, fused sparse Mix1: accumulator and x come back from tensor memory eight rows
+        // at a time, so that v / theta_new and the consensus sums are the only full-length arrays
+        float* const mom_col = a.momentum + (size_t)r0 * ld + col;
+        float* const new_col = a.theta_new + (size_t)r0 * ld + col;
+        float gh8[2][8], x8[2][8];                 // double-buffered: the next eight rows load while these compute
+        tmem_ld_8(tmem_acc + tmem_lane + (uint32_t)r0, gh8[0]);
+        tmem_ld_8(tmem_x, x8[0]);
+#pragma unroll
+        for (int mb = 0; mb < H; mb += 8) {
+          constexpr int kNext = 8;
+          const int cur = (mb / 8) & 1;
+          tmem_ld_wait();
+          if (mb + kNext < H) {
+            tmem_ld_8(tmem_acc + tmem_lane + (uint32_t)(r0 + mb + kNext), gh8[cur ^ 1]);
+            tmem_ld_8(tmem_x + (uint32_t)(mb + kNext), x8[cur ^ 1]);
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int m = mb + q;
+            const bool row_live = FULL || m < hr;
+            const float vn = fmaf(mu, v[m], gh8[cur][q]);
+            const float tn = fmaf(-lr, fmaf(mu, vn, gh8[cur][q]), x8[cur][q]);
+            if (live && row_live) {
+              __stcs(mom_col + (size_t)m * ld, vn);
+              __stcs(new_col + (size_t)m * ld, tn);
+            }
+            v[m] = tn;
+            asum += row_live ? tn : 0.f;
+          }
+        }
+      } else {
       float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
-      tmem_ld_cols<H>(tmem_acc + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, gh);
+      tmem_ld_cols<H>(tmem_acc + tmem_lane + (uint32_t)r0, gh);
       if constexpr (SUB) {
         if (!mix2_applies(a, col)) {
 #pragma unroll
@@ -363,7 +422,6 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         }
       }
       // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
-      float asum = 0.f;
       if (live) {
         float* const mom_col = a.momentum + (size_t)r0 * ld + col;
         float* const new_col = a.theta_new + (size_t)r0 * ld + col;
@@ -389,6 +447,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           asum += row_live ? tn : 0.f;
         }
       }
+      }
       if (want_cd || a.x_next) {                   // column mean over both halves, then squared deviations
         xchg[gid][h][c] = asum;
         named_bar_sync(3 + 3 * gid, CONS);
@@ -410,7 +469,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   __syncthreads();
   if (warp == ALLC / 32) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(NG * Shape::kTmemCols)) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemAll) : "memory");
   }
   if (want_cd) {
     double* red = reinterpret_cast<double*>(base);    // [ALLC/32][H]; per group: warps 0-3 hold the first half of the workers, 4-7 the second
