@@ -413,40 +413,40 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           }
         }
       } else {
-      float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
-      tmem_ld_cols<H>(tmem_acc + tmem_lane + (uint32_t)r0, gh);
-      if constexpr (SUB) {
-        if (!mix2_applies(a, col)) {
+        float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
+        tmem_ld_cols<H>(tmem_acc + tmem_lane + (uint32_t)r0, gh);
+        if constexpr (SUB) {
+          if (!mix2_applies(a, col)) {
 #pragma unroll
-          for (int m = 0; m < H; ++m) gh[m] = g[m];
+            for (int m = 0; m < H; ++m) gh[m] = g[m];
+          }
         }
-      }
-      // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
-      if (live) {
-        float* const mom_col = a.momentum + (size_t)r0 * ld + col;
-        float* const new_col = a.theta_new + (size_t)r0 * ld + col;
+        // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
+        if (live) {
+          float* const mom_col = a.momentum + (size_t)r0 * ld + col;
+          float* const new_col = a.theta_new + (size_t)r0 * ld + col;
 #pragma unroll
-        for (int m = 0; m < H; ++m) {
-          // With a per-row x the padded rows are computed like the others (their inputs are zeros)
-          // and only kept out of the stores and of the column sum: an early exit from the unrolled
-          // loop cost those register-heavy variants half their speed.  Without one it is the
-          // faster form.
-          if constexpr (!XMAT) {
-            if (!FULL && m >= hr) break;
+          for (int m = 0; m < H; ++m) {
+            // With a per-row x the padded rows are computed like the others (their inputs are zeros)
+            // and only kept out of the stores and of the column sum: an early exit from the unrolled
+            // loop cost those register-heavy variants half their speed.  Without one it is the
+            // faster form.
+            if constexpr (!XMAT) {
+              if (!FULL && m >= hr) break;
+            }
+            const bool row_live = FULL || m < hr;
+            const float vn = fmaf(mu, v[m], gh[m]);
+            float xm = xv;
+            if constexpr (XMAT) xm = xr[m];
+            const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xm);
+            if (row_live) {
+              __stcs(mom_col + (size_t)m * ld, vn);
+              __stcs(new_col + (size_t)m * ld, tn);
+            }
+            v[m] = tn;
+            asum += row_live ? tn : 0.f;
           }
-          const bool row_live = FULL || m < hr;
-          const float vn = fmaf(mu, v[m], gh[m]);
-          float xm = xv;
-          if constexpr (XMAT) xm = xr[m];
-          const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xm);
-          if (row_live) {
-            __stcs(mom_col + (size_t)m * ld, vn);
-            __stcs(new_col + (size_t)m * ld, tn);
-          }
-          v[m] = tn;
-          asum += row_live ? tn : 0.f;
         }
-      }
       }
       if (want_cd || a.x_next) {                   // column mean over both halves, then squared deviations
         xchg[gid][h][c] = asum;
