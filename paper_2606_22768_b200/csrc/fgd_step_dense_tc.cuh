@@ -170,10 +170,11 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
   constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
   constexpr int ALLC = NG * CONS;                   // all consumer threads; the producer warp follows them
-  // tensor memory: the accumulator columns of every group, then (fused sparse Mix1) as many scratch
-  // columns for x; 32 + 32, 64 + 64: powers of two
-  constexpr int kTmemAll = NG * Shape::kTmemCols + (XM == 2 ? Shape::kTmemCols : 0);
-  static_assert(XM != 2 || NG == 1, "the x scratch columns are laid out for one consumer group");
+  // tensor memory: the accumulator columns of every group, then as many scratch columns: x of a
+  // fused sparse Mix1, or g where Mix2 is restricted to column ranges; 32 + 32, 64 + 64: powers of two
+  constexpr int kTmemAll = NG * Shape::kTmemCols + ((XM == 2 || SUB) ? Shape::kTmemCols : 0);
+  static_assert(!(XM == 2 || SUB) || NG == 1, "the scratch columns are laid out for one consumer group");
+  static_assert(!(XM == 2 && SUB), "one set of scratch columns");
   static_assert(STAGES % NG == 0, "every stage belongs to one group");
   const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -268,7 +269,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     const int lt = tid & (CONS - 1);              // index within the group
     const int c = lt & (T - 1), h = lt >> 7, r0 = h * H;
     const uint32_t tmem_lane = (uint32_t)((warp & 3) * 32) << 16;      // this warp's quarter of the lanes
-    // scratch columns of this thread for a fused sparse Mix1 result (behind all accumulator columns)
+    // scratch columns of this thread (behind all accumulator columns)
     const uint32_t tmem_x = tmem_base + (uint32_t)(NG * Shape::kTmemCols) + tmem_lane + (uint32_t)r0;
     const float invK = 1.0f / (float)KR;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
@@ -311,6 +312,11 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           tsum += tp;
         }
         if (need_tsum) xsum[gid][h][c] = tsum;          // the column mean needs the other half's sum too
+        if constexpr (SUB) {                       // outside the ranges ghat = g: park g next to the accumulator
+#pragma unroll
+          for (int n = 0; n < H; n += 8) tmem_st_8(tmem_x + (uint32_t)n, &g[n]);
+          tmem_st_wait();
+        }
         if constexpr (XM == 2) {                   // gossip Mix1 of this thread's rows, from the stage
           const int D1 = m1.D;                     // (uniform) -> a fully unrolled gather per slot count
           if (D1 == 0) tc_gather_x<0, H, T>(m1, A, r0, c, tmem_x);
@@ -414,12 +420,25 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         }
       } else {
         float gh[H];                                 // TMEM lane = column, TMEM columns r0.. = this thread's workers
-        tmem_ld_cols<H>(tmem_acc + tmem_lane + (uint32_t)r0, gh);
         if constexpr (SUB) {
-          if (!mix2_applies(a, col)) {
+          // identity on a column outside the ranges: read g back instead of W g.  A tensor-memory
+          // load takes ONE address per warp, so the choice is made per warp; the rare warp that
+          // straddles a range boundary reads both and selects per thread.
+          const bool applies = mix2_applies(a, col);
+          const bool any_in = __any_sync(0xffffffffu, applies), all_in = __all_sync(0xffffffffu, applies);
+          tmem_ld_cols<H>(any_in ? tmem_acc + tmem_lane + (uint32_t)r0 : tmem_x, gh);
+          if (any_in && !all_in) {
 #pragma unroll
-            for (int m = 0; m < H; ++m) gh[m] = g[m];
+            for (int n = 0; n < H; n += 8) {
+              float t8[8];
+              tmem_ld_8(tmem_x + (uint32_t)n, t8);
+              tmem_ld_wait();
+#pragma unroll
+              for (int q = 0; q < 8; ++q) gh[n + q] = applies ? gh[n + q] : t8[q];
+            }
           }
+        } else {
+          tmem_ld_cols<H>(tmem_acc + tmem_lane + (uint32_t)r0, gh);
         }
         // ---- phase 2: Nesterov step for this thread's workers of the column, stream out
         if (live) {
