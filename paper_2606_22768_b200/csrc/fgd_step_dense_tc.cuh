@@ -161,12 +161,11 @@ __device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A,
 // (registers are handed out per four warps: 288 threads count as 384, i.e. at most 168 registers
 // each, and 544 as 640, i.e. 96 -- asking for more makes the kernel unlaunchable)
 template <int KP, int XM, bool FULL, bool SUB = false, int NG = 1>
-__global__ void __launch_bounds__(NG * kTcConsumers + 32)
+__global__ void __launch_bounds__(NG * kTcConsumers + 32, 1)
 outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const GatherMix m1,
                            const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                            const __grid_constant__ CUtensorMap tm_mom, const __grid_constant__ CUtensorMap tm_x) {
   using Shape = TcShape<KP>;
-  constexpr bool XMAT = XM != 0;                    // x differs from row to row
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = Shape::kStages;
   constexpr uint32_t kTcBox = Shape::kBox, kTcWBytes = Shape::kWBytes, SBO = Shape::kSbo;
   constexpr int ALLC = NG * CONS;                   // all consumer threads; the producer warp follows them
@@ -387,14 +386,15 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       mbar_arrive(smem_u32(&bars[STAGES + s]));
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float asum = 0.f;
-      if constexpr (XM == 2) {
-        // ---- phase 2, fused sparse Mix1: accumulator and x come back from tensor memory eight rows
-        // at a time, so that v / theta_new and the consensus sums are the only full-length arrays
+      if constexpr (XM != 0) {
+        // ---- phase 2, per-row x: the accumulator (and the x of a fused sparse Mix1) comes back from
+        // tensor memory eight rows at a time, which keeps the full-length register arrays to v /
+        // theta_new, the consensus sums and -- for a matrix-valued x -- the prefetched x itself
         float* const mom_col = a.momentum + (size_t)r0 * ld + col;
         float* const new_col = a.theta_new + (size_t)r0 * ld + col;
         float gh8[2][8], x8[2][8];                 // double-buffered: the next eight rows load while these compute
         tmem_ld_8(tmem_acc + tmem_lane + (uint32_t)r0, gh8[0]);
-        tmem_ld_8(tmem_x, x8[0]);
+        if constexpr (XM == 2) tmem_ld_8(tmem_x, x8[0]);
 #pragma unroll
         for (int mb = 0; mb < H; mb += 8) {
           constexpr int kNext = 8;
@@ -402,14 +402,17 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           tmem_ld_wait();
           if (mb + kNext < H) {
             tmem_ld_8(tmem_acc + tmem_lane + (uint32_t)(r0 + mb + kNext), gh8[cur ^ 1]);
-            tmem_ld_8(tmem_x + (uint32_t)(mb + kNext), x8[cur ^ 1]);
+            if constexpr (XM == 2) tmem_ld_8(tmem_x + (uint32_t)(mb + kNext), x8[cur ^ 1]);
           }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const int m = mb + q;
             const bool row_live = FULL || m < hr;
             const float vn = fmaf(mu, v[m], gh8[cur][q]);
-            const float tn = fmaf(-lr, fmaf(mu, vn, gh8[cur][q]), x8[cur][q]);
+            float xq;
+            if constexpr (XM == 2) xq = x8[cur][q];
+            else xq = xr[m];
+            const float tn = fmaf(-lr, fmaf(mu, vn, gh8[cur][q]), xq);
             if (live && row_live) {
               __stcs(mom_col + (size_t)m * ld, vn);
               __stcs(new_col + (size_t)m * ld, tn);
@@ -446,24 +449,13 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
           float* const new_col = a.theta_new + (size_t)r0 * ld + col;
 #pragma unroll
           for (int m = 0; m < H; ++m) {
-            // With a per-row x the padded rows are computed like the others (their inputs are zeros)
-            // and only kept out of the stores and of the column sum: an early exit from the unrolled
-            // loop cost those register-heavy variants half their speed.  Without one it is the
-            // faster form.
-            if constexpr (!XMAT) {
-              if (!FULL && m >= hr) break;
-            }
-            const bool row_live = FULL || m < hr;
-            const float vn = fmaf(mu, v[m], gh[m]);
-            float xm = xv;
-            if constexpr (XMAT) xm = xr[m];
-            const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xm);
-            if (row_live) {
-              __stcs(mom_col + (size_t)m * ld, vn);
-              __stcs(new_col + (size_t)m * ld, tn);
-            }
+            if (!FULL && m >= hr) break;           // (the per-row-x branch above predicates instead: an
+            const float vn = fmaf(mu, v[m], gh[m]);  //  early exit cost those register-heavy variants half their speed)
+            const float tn = fmaf(-lr, fmaf(mu, vn, gh[m]), xv);
+            __stcs(mom_col + (size_t)m * ld, vn);
+            __stcs(new_col + (size_t)m * ld, tn);
             v[m] = tn;
-            asum += row_live ? tn : 0.f;
+            asum += tn;
           }
         }
       }
