@@ -149,3 +149,50 @@ def test_more_than_2_to_31_columns():
     assert e.value.status == fgd.FGD_ERR_UNSUPPORTED
     del theta, local, mom
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("K,P,mix1,fused", [(40, 40_000_037, ("mean",), False),      # padded to 48 workers, ragged tail
+                                            (56, 30_000_004, ("ring", 0.1), True),   # padded to 64, gossip Mix1 fused
+                                            (12, 100_000_002, ("ring",), False)])    # compile-time 12, matrix-valued x
+def test_full_size_other_worker_counts(K, P, mix1, fused):
+    """Worker counts beside the benchmark configurations at sizes of many thousand tiles per CTA:
+    zero-padded tensor-core shapes and the 12-worker kernel, 3 free-running rounds, sampled blocks."""
+    seed = 21
+    ld = (P + 3) // 4 * 4
+    need = 4 * K * ld * 4 + (2 << 30)
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip("not enough free HBM for this size")
+    sig = np.full(K, 1e-3, np.float32)
+    full = [torch.full((K, ld), -777.0, dtype=torch.float32, device="cuda") for _ in range(3)]
+    theta, local, mom = (t[:, :P] for t in full)
+    inputs_gpu.theta0(theta, seed)
+    mom.zero_()
+    drv = OuterRound(K, P, ld)
+    blocks = sorted({0, P - WIDTH, 127 * 1000 + 5, (P // 2) // 128 * 128 - 40, P // 3})
+    o_theta = {p0: gen.theta0(seed, K, P, p0=p0, p1=p0 + WIDTH).astype(np.float64) for p0 in blocks}
+    o_v = {p0: np.zeros((K, WIDTH)) for p0 in blocks}
+    cd_alone = torch.zeros(K, dtype=torch.float64, device="cuda")
+    for r in range(3):
+        d1, W1 = make_mix(mix1, K, r, seed, 1)
+        d2, W2 = make_mix(("ring", 0.2), K, r, seed, 2)
+        inputs_gpu.local_steps(local, theta, sig, seed, r)
+        if fused:
+            drv.step(d2, full[1], full[0], full[2], full[0], 0.7, 0.9, mix1_fused=d1)
+        else:
+            drv.launch_mix1(d1, full[0])
+            drv.step(d2, full[1], full[0], full[2], full[0], 0.7, 0.9)
+        fgd.fgd_consensus_distance(drv.ctx, full[0], cd_alone)
+        torch.cuda.synchronize()
+        fused_cd, alone = drv.cd_sumsq.cpu().numpy(), cd_alone.cpu().numpy()
+        assert np.all(np.abs(fused_cd - alone) <= 2e-6 * np.abs(alone)), f"round {r}: fused {fused_cd} vs stand-alone {alone}"
+        for p0 in blocks:
+            drift = gen.scaled_normal(seed, gen.TENSOR_DRIFT, r, K, P, sig, p0, p0 + WIDTH).astype(np.float64)
+            o_theta[p0], o_v[p0] = oracle.outer_round(W1, W2, o_theta[p0], o_theta[p0] + drift, o_v[p0], 0.7, 0.9)
+            assert_param_close(theta[:, p0:p0 + WIDTH], o_theta[p0], f"K={K} round {r} theta_new block {p0}")
+            assert_param_close(mom[:, p0:p0 + WIDTH], o_v[p0], f"K={K} round {r} momentum block {p0}")
+    fgd.fgd_device_status(drv.ctx)
+    for t in full:
+        if ld > P:
+            assert bool((t[:, P:] == -777.0).all()), "padding columns were written"
+    del theta, local, mom, full
+    torch.cuda.empty_cache()
