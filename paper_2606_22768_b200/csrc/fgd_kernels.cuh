@@ -751,7 +751,8 @@ mix_mean_split_kernel(const float* __restrict__ in, float* __restrict__ out, int
 }
 
 // out[m] = sum_b partials[b][m], fixed order: one warp per worker, lanes stride the blocks,
-// then a shuffle tree.  Deterministic.
+// then a shuffle tree.  Deterministic.  The same sum as finalize_in_last_cta, as a launch of its
+// own: used by the allocation-free entry point, which has no finished-CTA counter.
 static __global__ void __launch_bounds__(32)
 consensus_finalize_kernel(const double* __restrict__ partials, int nblocks, int K, double* __restrict__ out) {
   const int m = blockIdx.x, lane = threadIdx.x;
