@@ -447,3 +447,15 @@ def test_argument_errors():
     # the context is still usable after errors
     fgd.fgd_outer_grad(ctx, a, b, c)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("K,P,mix1,mix2,rounds", [
+    (8, 20000, ("mean",), ("matching", 0.05), 60),                          # the paper's setting, many rounds
+    (64, 6000, ("ring", 0.1), ("dense", gen.sinkhorn_W(0, 64)), 30),        # tensor-core step and mix
+    (48, 5000, ("mean",), ("ring",), 40),                                   # padded tensor-core shape
+])
+def test_long_free_running_rounds(K, P, mix1, mix2, rounds):
+    """Many free-running rounds (the oracle keeps its own float64 state): the fp32 path must not drift
+    out of tolerance -- nothing accumulates beyond rounding, as a contraction with a doubly stochastic
+    matrix cannot amplify it."""
+    Scenario(K, P, mix1, mix2, seed=3, mode="factored").run(rounds)
