@@ -313,10 +313,11 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   // is the fastest fused step we have there, and any mix is also a dense matrix -- so a gather /
   // mean Mix2 is densified and takes it too.
   // K = 32 has a compile-time fp32 kernel that is the faster one for a light sparse Mix2 (at most two
-  // neighbour slots) with x one value per column or gathered in the kernel (ring: 5.8 / 5.1 TB/s
-  // against 5.6 / 4.9); with more slots (hypercube: 2.4 TB/s against 5.6) or a matrix-valued x
-  // (5.1 against 5.8) the tensor-core kernel wins.
-  const bool tc_at_32 = dense2 || (g2.kind == KMIX_GATHER && g2.D > 2) || a.xsrc == XSRC_MATRIX;
+  // neighbour slots) with x one value per column (ring: 5.8 TB/s against 5.6); with more slots
+  // (hypercube: 2.4 TB/s against 5.6), a matrix-valued x (5.1 against 5.8) or a sparse Mix1 gathered
+  // in the kernel (5.1 against 5.4) the tensor-core kernel wins.
+  const bool tc_at_32 = dense2 || (g2.kind == KMIX_GATHER && g2.D > 2) || a.xsrc == XSRC_MATRIX ||
+                        (a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER);
   bool can_tc = c->path != FGD_PATH_TMA_FP32 && fgd_tc_eligible(c, a, tc_at_32, g1);
   if (can_tc && !dense2) {
     double Wd[FGD_MAX_K * FGD_MAX_K];

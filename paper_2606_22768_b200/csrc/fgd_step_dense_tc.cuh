@@ -171,8 +171,8 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
   constexpr int ALLC = NG * CONS;                   // all consumer threads; the producer warp follows them
   // tensor memory: the accumulator columns of every group, then as many scratch columns: x of a
   // fused sparse Mix1, or g where Mix2 is restricted to column ranges; 32 + 32, 64 + 64: powers of two
-  constexpr int kTmemAll = NG * Shape::kTmemCols + ((XM == 2 || SUB) ? Shape::kTmemCols : 0);
-  static_assert(!(XM == 2 || SUB) || NG == 1, "the scratch columns are laid out for one consumer group");
+  constexpr int kTmemAll = NG * Shape::kTmemCols * ((XM == 2 || SUB) ? 2 : 1);   // per group: accumulator [+ scratch]
+  static_assert(kTmemAll <= 128, "tensor-memory budget of this kernel");
   static_assert(!(XM == 2 && SUB), "one set of scratch columns");
   static_assert(STAGES % NG == 0, "every stage belongs to one group");
   const int KR = FULL ? K : ta.s.K;                 // real worker count (<= K)
@@ -269,7 +269,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     const int c = lt & (T - 1), h = lt >> 7, r0 = h * H;
     const uint32_t tmem_lane = (uint32_t)((warp & 3) * 32) << 16;      // this warp's quarter of the lanes
     // scratch columns of this thread (behind all accumulator columns)
-    const uint32_t tmem_x = tmem_base + (uint32_t)(NG * Shape::kTmemCols) + tmem_lane + (uint32_t)r0;
+    const uint32_t tmem_x = tmem_base + (uint32_t)((NG + gid) * Shape::kTmemCols) + tmem_lane + (uint32_t)r0;
     const float invK = 1.0f / (float)KR;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);   // live workers of this thread
     const float lr = a.lr, mu = a.mu;

@@ -52,7 +52,11 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
   const int xm = a.xsrc == XSRC_MATRIX ? 1 : ((a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER) ? 2 : 0);
   switch (xm) {
     case 1: return full ? launch(outer_step_dense_tc_kernel<KP, 1, true>) : launch(outer_step_dense_tc_kernel<KP, 1, false>);
-    case 2: return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
+    case 2:
+      if constexpr (KP == 32)    // two consumer groups where the registers allow it
+        return full ? launch(outer_step_dense_tc_kernel<KP, 2, true, false, 2>, 2) : launch(outer_step_dense_tc_kernel<KP, 2, false, false, 2>, 2);
+      else
+        return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
     default:
       if (a.n_ranges != 0)
         return full ? launch(outer_step_dense_tc_kernel<KP, 0, true, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false, true>);
