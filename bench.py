@@ -55,7 +55,8 @@ CONFIGS = {
 # DRAM bytes per worker-parameter of the fused outer-step kernel measured with ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch / (K*P) of that launch); the
 # capture it comes from is summarised under profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {3: 20.04, 5: 19.85}
+NCU_TRAFFIC_BYTES_PER_WORKER_PARAM = {2: 20.29, 3: 20.04, 4: 23.81, 5: 19.85, 6: 20.29}   # 6 runs config 2's kernel
+NCU_TRAFFIC_FUSED_MIX1 = {4: 19.79}   # the same with --fuse-mix1
 
 
 def parse_args():
@@ -369,7 +370,9 @@ def run_ours(args):
         step_bytes, mix1_bytes = 20 * K * P, 0
     peak, peak_kind = measured_peak()
     achieved = step_bytes / (kern_ms * 1e-3) / 1e9
-    tr = NCU_TRAFFIC_BYTES_PER_WORKER_PARAM.get(args.config)
+    tr = (NCU_TRAFFIC_FUSED_MIX1 if args.fuse_mix1 else NCU_TRAFFIC_BYTES_PER_WORKER_PARAM).get(args.config)
+    if args.subset_frac > 0.0 or args.average_momentum or args.chain_mix1 or args.graph:
+        tr = None                   # variants were not captured
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if tr is None else tr * K * P,
                 "kernel": "outer_step_dense_tc_kernel" if K == 64 else "outer_step_tma_kernel",
