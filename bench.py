@@ -614,24 +614,26 @@ def latency_leg(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, dev, rep
     return out
 
 
-def e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W, world, dev, steps=3):
-    """Same round with theta_local arriving from pinned HOST memory every step and the consensus
-    sums read back to the host every step (both inside the timed region)."""
+def e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W, world, dev, steps=3, n_chunks=16):
+    """Same round through the C-ABI call that takes theta_local from HOST memory
+    (fgd_outer_step_from_host: pinned host matrix, copied in column chunks that overlap the fused
+    step of the previous chunk) and returns the consensus sums to the host; both transfers are
+    inside the timed region, every step."""
     K, P = cfg["K"], cfg["P"]
     host_local = torch.empty((K, P), dtype=torch.float32, pin_memory=True)
     host_local.copy_(local)
-    host_cd = torch.empty(K, dtype=torch.float64, pin_memory=True)
     main = torch.cuda.current_stream(dev)
 
     def one(r):
         m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
         m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
-        drv.cd_sumsq = cd_log[0]
-        drv.launch_mix1(m1, theta)                       # overlaps the host-to-device copy
-        local.copy_(host_local, non_blocking=True)
-        drv.step(m2, local, theta, mom, theta, 0.7, 0.9)
-        host_cd.copy_(cd_log[0], non_blocking=True)
-        main.synchronize()
+        drv.launch_mix1(m1, theta)                       # side stream: overlaps the first chunk's copy
+        ev, x, is_vec = drv._pending
+        drv._pending = None
+        main.wait_event(ev)
+        fgd.fgd_outer_step_from_host(drv.ctx, m2, None, x, is_vec, host_local, local, theta, mom, theta, 0.7, 0.9,
+                                     want_cd=True, n_chunks=n_chunks)   # returns once the sums are on the host
+        drv.side.wait_event(main.record_event())          # x may be overwritten by the next round's Mix1 only now
 
     one(0)
     torch.cuda.synchronize()
@@ -646,7 +648,8 @@ def e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W
     ms = a.elapsed_time(b)
     ms, units = aggregate(dist if world > 1 else None, ms, K * P, dev)
     return {"value": units / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": K * P * 4,
-            "d2h_bytes_per_step": K * 8, "steps": steps, "ms_per_step": ms / steps}
+            "d2h_bytes_per_step": K * 8 * min(n_chunks, (P + 1023) // 1024), "steps": steps, "ms_per_step": ms / steps,
+            "call": f"fgd_outer_step_from_host, {n_chunks} column chunks"}
 
 
 def main():

@@ -56,6 +56,7 @@ extern "C" {
 #define FGD_MAX_K 64 /* most workers (rows) */
 #define FGD_MAX_D 8  /* most neighbour slots per worker in a sparse mix */
 #define FGD_MAX_RANGES 8 /* most column ranges of a subset Mix2 */
+#define FGD_MAX_CHUNKS 32 /* most column chunks of fgd_outer_step_from_host */
 
 typedef enum {
   FGD_OK = 0,
@@ -187,6 +188,24 @@ int fgd_outer_step_ex(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc
                       const float* x, int x_is_vector, const float* theta_local,
                       const float* theta_prev, float* momentum, float* theta_new, double lr,
                       double mu, double* cd_sumsq, const fgd_step_options* opts, void* stream);
+
+/* The same outer step (Algorithm 1, the blocking part of the round) when the inner steps'
+ * result arrives from HOST memory: theta_local_host is a HOST [K, ld] matrix (pinned memory
+ * for full copy bandwidth; pageable works, more slowly), theta_local_dev a DEVICE [K, ld]
+ * staging matrix of the caller.  The columns are cut into n_chunks (1..FGD_MAX_CHUNKS) chunks
+ * on 1024-column boundaries; chunk i+1 is copied on an internal stream while the fused step
+ * of chunk i runs on `stream` (columns are independent, so the result is that of
+ * fgd_outer_step on the whole matrix, bit for bit in theta_new and momentum).  cd_sumsq_host:
+ * HOST [K] doubles or NULL; the per-chunk sums are added in chunk order.  No mix2_ranges /
+ * momentum averaging here.  Unlike the other calls this one RETURNS AFTER THE ROUND HAS
+ * COMPLETED on the device when cd_sumsq_host is given (it has to read the sums back);
+ * with NULL it is asynchronous like the rest.  The first call creates the internal stream,
+ * events and 32 KB of device and pinned host memory (so: not inside a stream capture). */
+int fgd_outer_step_from_host(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused,
+                             const float* x, int x_is_vector, const float* theta_local_host,
+                             float* theta_local_dev, const float* theta_prev, float* momentum,
+                             float* theta_new, double lr, double mu, double* cd_sumsq_host,
+                             int n_chunks, void* stream);
 
 /* s_m = sum_p (theta[m][p] - (1/K) sum_n theta[n][p])^2 into device cd_sumsq[K] (doubles).
  * The paper gives two L2 consensus distances, both functions of s: the mean of the

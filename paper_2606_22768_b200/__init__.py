@@ -69,6 +69,7 @@ def _load():
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
         "fgd_outer_step_ex": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp, vp]),
+        "fgd_outer_step_from_host": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, vp, dbl, dbl, vp, i32, vp]),
         "fgd_consensus_distance": (i32, [vp, vp, vp, vp]),
         "fgd_consensus_distance_noalloc": (i32, [i32, i32, i64, i64, vp, vp, vp]),
         "fgd_js_distance": (i32, [i32, i32, i64, i64, i32, vp, vp, vp, vp, vp, vp]),
@@ -330,6 +331,31 @@ def fgd_outer_step_ex(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc]
         _dev_ptr(momentum, "momentum", "torch.float32"),
         _dev_ptr(theta_new, "theta_new", "torch.float32"), float(lr), float(mu),
         _dev_ptr(cd_sumsq, "cd_sumsq", "torch.float64"), ctypes.byref(opts), _stream(stream)))
+
+
+def fgd_outer_step_from_host(ctx: Context, mix2: MixDesc, mix1_fused: Optional[MixDesc], x, x_is_vector: bool,
+                             theta_local_host, theta_local_dev, theta_prev, momentum, theta_new,
+                             lr: float = 0.7, mu: float = 0.9, want_cd: bool = True, n_chunks: int = 8,
+                             stream=None) -> Optional[np.ndarray]:
+    """The outer step with theta_local arriving from HOST memory (a CPU tensor [K, ld], pinned for
+    full copy bandwidth): copied chunk by chunk into ``theta_local_dev`` while the previous chunk's
+    step runs.  With ``want_cd`` the call returns the consensus sums (float64 [K]) after the round
+    has completed; without it returns None and is asynchronous."""
+    if getattr(theta_local_host, "is_cuda", True) or str(theta_local_host.dtype) != "torch.float32":
+        raise TypeError("theta_local_host must be a float32 CPU tensor")
+    if theta_local_host.stride(-1) != 1 or (theta_local_host.dim() == 2 and theta_local_host.shape[0] > 1
+                                             and theta_local_host.stride(0) != ctx.ld):
+        raise ValueError("theta_local_host must be a [K, ld] matrix with the context's row stride")
+    cd = np.empty(ctx.K, dtype=np.float64) if want_cd else None
+    ctx._check(_lib.fgd_outer_step_from_host(
+        ctx._h, ctypes.byref(mix2.c()), None if mix1_fused is None else ctypes.byref(mix1_fused.c()),
+        _dev_ptr(x, "x", "torch.float32"), int(bool(x_is_vector)), theta_local_host.data_ptr(),
+        _dev_ptr(theta_local_dev, "theta_local_dev", "torch.float32"),
+        _dev_ptr(theta_prev, "theta_prev", "torch.float32"),
+        _dev_ptr(momentum, "momentum", "torch.float32"),
+        _dev_ptr(theta_new, "theta_new", "torch.float32"), float(lr), float(mu),
+        None if cd is None else cd.ctypes.data, int(n_chunks), _stream(stream)))
+    return cd
 
 
 def fgd_consensus_distance(ctx: Context, theta, cd_sumsq, stream=None) -> None:

@@ -36,6 +36,13 @@ struct fgd_ctx {
   int64_t launches = 0;
   char err[256] = "";
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
+  // fgd_outer_step_from_host only (created by its first call): copy stream, one event per column
+  // chunk, per-chunk consensus sums on the device and their pinned host copy
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t start_ev = nullptr;
+  cudaEvent_t chunk_ev[FGD_MAX_CHUNKS] = {};
+  double* chunk_cd = nullptr;       // device [FGD_MAX_CHUNKS][FGD_MAX_K]
+  double* chunk_cd_host = nullptr;  // pinned host, same shape
 };
 
 namespace {
