@@ -34,6 +34,9 @@
  *  - Fast path: base pointers 16-byte aligned and ld % 4 == 0; otherwise an element-wise
  *    path is used (slower, not an error).
  *  - Deterministic: the same inputs give bit-identical outputs (no floating-point atomics).
+ *  - Threads: a context is NOT re-entrant.  It carries the last error string, an occupancy cache
+ *    and (during fgd_outer_step_from_host) a temporarily narrowed column count, so one context
+ *    must be used by one host thread at a time; different contexts are independent.
  *  - fgd_outer_step (with cd_sumsq) and fgd_consensus_distance use the context's small
  *    partial-sum scratch: two such calls on one context must be ordered on the GPU
  *    (same stream or an event); all other calls may overlap freely.
@@ -199,8 +202,12 @@ int fgd_outer_step_ex(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc
  * HOST [K] doubles or NULL; the per-chunk sums are added in chunk order.  No mix2_ranges /
  * momentum averaging here.  Unlike the other calls this one RETURNS AFTER THE ROUND HAS
  * COMPLETED on the device when cd_sumsq_host is given (it has to read the sums back);
- * with NULL it is asynchronous like the rest.  The first call creates the internal stream,
- * events and 32 KB of device and pinned host memory (so: not inside a stream capture). */
+ * with NULL it is asynchronous like the rest.  Only the K consensus doubles come back to the
+ * host: theta_new and the momentum stay on the device, where the next round reads them.  The
+ * first call creates the internal stream, events and 32 KB of device and pinned host memory (so:
+ * not inside a stream capture); if that set-up fails the call returns FGD_ERR_CUDA before any
+ * launch and the next call tries again.  While the call runs it narrows the context's column
+ * count to the chunk it is launching: no other thread may use this context meanwhile. */
 int fgd_outer_step_from_host(fgd_ctx* ctx, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused,
                              const float* x, int x_is_vector, const float* theta_local_host,
                              float* theta_local_dev, const float* theta_prev, float* momentum,

@@ -60,14 +60,13 @@ int fgd_destroy(fgd_ctx* c) {
   cudaError_t e = cudaFree(c->partials);
   cudaFree(c->status);
   cudaFree(c->done);
-  if (c->copy_stream) {   // resources of fgd_outer_step_from_host
-    cudaStreamDestroy(c->copy_stream);
-    if (c->start_ev) cudaEventDestroy(c->start_ev);
-    for (cudaEvent_t ev : c->chunk_ev)
-      if (ev) cudaEventDestroy(ev);
-    cudaFree(c->chunk_cd);
-    cudaFreeHost(c->chunk_cd_host);
-  }
+  // resources of fgd_outer_step_from_host (all present or all null)
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->start_ev) cudaEventDestroy(c->start_ev);
+  for (cudaEvent_t ev : c->chunk_ev)
+    if (ev) cudaEventDestroy(ev);
+  if (c->chunk_cd) cudaFree(c->chunk_cd);
+  if (c->chunk_cd_host) cudaFreeHost(c->chunk_cd_host);
   delete c;
   return e == cudaSuccess ? FGD_OK : cuda_fail(nullptr, e, "fgd_destroy");
 }

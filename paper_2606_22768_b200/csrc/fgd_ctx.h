@@ -38,6 +38,7 @@ struct fgd_ctx {
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
   // fgd_outer_step_from_host only (created by its first call): copy stream, one event per column
   // chunk, per-chunk consensus sums on the device and their pinned host copy
+  bool streaming_ready = false;     // all of the below exist (set only after every one was created)
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t start_ev = nullptr;
   cudaEvent_t chunk_ev[FGD_MAX_CHUNKS] = {};

@@ -7,15 +7,52 @@
 
 namespace {
 
+// Frees whatever the streaming set-up has created so far and leaves every handle null.
+void release_streaming_resources(fgd_ctx* c) {
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->start_ev) cudaEventDestroy(c->start_ev);
+  for (cudaEvent_t& ev : c->chunk_ev) {
+    if (ev) cudaEventDestroy(ev);
+    ev = nullptr;
+  }
+  if (c->chunk_cd) cudaFree(c->chunk_cd);
+  if (c->chunk_cd_host) cudaFreeHost(c->chunk_cd_host);
+  c->copy_stream = nullptr;
+  c->start_ev = nullptr;
+  c->chunk_cd = nullptr;
+  c->chunk_cd_host = nullptr;
+  c->streaming_ready = false;
+}
+
+// Creates the copy stream, the events and the two small consensus buffers.  All or nothing: when
+// any step fails everything made so far is released again, so a later call starts from scratch
+// instead of running with a missing buffer.
 int ensure_streaming_resources(fgd_ctx* c) {
-  if (c->copy_stream) return FGD_OK;
-  FGD_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
-  FGD_CUDA(c, cudaEventCreateWithFlags(&c->start_ev, cudaEventDisableTiming));
-  for (int i = 0; i < FGD_MAX_CHUNKS; ++i) FGD_CUDA(c, cudaEventCreateWithFlags(&c->chunk_ev[i], cudaEventDisableTiming));
-  FGD_CUDA(c, cudaMalloc(&c->chunk_cd, sizeof(double) * FGD_MAX_CHUNKS * FGD_MAX_K));
-  FGD_CUDA(c, cudaMallocHost(&c->chunk_cd_host, sizeof(double) * FGD_MAX_CHUNKS * FGD_MAX_K));
+  if (c->streaming_ready) return FGD_OK;
+  cudaError_t e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->start_ev, cudaEventDisableTiming);
+  for (int i = 0; i < FGD_MAX_CHUNKS && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->chunk_ev[i], cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaMalloc(&c->chunk_cd, sizeof(double) * FGD_MAX_CHUNKS * FGD_MAX_K);
+  if (e == cudaSuccess) e = cudaMallocHost(&c->chunk_cd_host, sizeof(double) * FGD_MAX_CHUNKS * FGD_MAX_K);
+  if (e != cudaSuccess || !c->copy_stream || !c->start_ev || !c->chunk_cd || !c->chunk_cd_host) {
+    release_streaming_resources(c);
+    cudaGetLastError();
+    return fail(c, FGD_ERR_CUDA, "fgd_outer_step_from_host: set-up of the copy stream and buffers failed: %s",
+                e != cudaSuccess ? cudaGetErrorString(e) : "a handle is missing");
+  }
+  c->streaming_ready = true;
   return FGD_OK;
 }
+
+// The step of one column window runs through the ordinary entry point with the context's column
+// count narrowed to the window (same row stride); restored on every exit path.  This is why a
+// context must not be shared between threads while this call runs.
+struct ColumnWindow {
+  fgd_ctx* c;
+  int64_t saved;
+  ColumnWindow(fgd_ctx* ctx, int64_t cols) : c(ctx), saved(ctx->P) { c->P = cols; }
+  ~ColumnWindow() { c->P = saved; }
+};
 
 }  // namespace
 
@@ -54,11 +91,10 @@ extern "C" int fgd_outer_step_from_host(fgd_ctx* c, const fgd_mix_desc* mix2, co
   for (int i = 0; i < n && rc == FGD_OK; ++i) {
     const int64_t c0 = (int64_t)i * w, c1 = c0 + w < P ? c0 + w : P;
     FGD_CUDA(c, cudaStreamWaitEvent(st, c->chunk_ev[i], 0));
-    c->P = c1 - c0;   // the window [c0, c1) of every matrix: same row stride, fewer columns
+    ColumnWindow window(c, c1 - c0);   // the window [c0, c1) of every matrix: same row stride, fewer columns
     rc = fgd_outer_step_ex(c, mix2, mix1_fused, x ? x + c0 : nullptr, x_is_vector, theta_local_dev + c0, theta_prev + c0,
                            momentum + c0, theta_new + c0, lr, mu, cd_sumsq_host ? c->chunk_cd + (size_t)i * K : nullptr,
                            nullptr, st);
-    c->P = P;
   }
   if (rc != FGD_OK) return rc;
   if (cd_sumsq_host) {

@@ -93,6 +93,12 @@ extern "C" int fgd_consensus_distance_noalloc(int device, int K, int64_t P, int6
                    kNoAllocBlocks, FGD_MAX_K, FGD_MAX_K);
   if (P < 1 || ld < P) return na_fail(FGD_ERR_INVALID_ARG, "need 1 <= P <= ld (P=%lld, ld=%lld)", (long long)P, (long long)ld);
   if (!theta || !cd_sumsq) return na_fail(FGD_ERR_INVALID_ARG, "NULL pointer");
+  {  // the K output doubles must not lie inside the matrix they are computed from
+    const uintptr_t t_lo = reinterpret_cast<uintptr_t>(theta);
+    const uintptr_t t_hi = t_lo + (uintptr_t)(((int64_t)(K - 1) * ld + P) * (int64_t)sizeof(float));
+    const uintptr_t o_lo = reinterpret_cast<uintptr_t>(cd_sumsq), o_hi = o_lo + (uintptr_t)K * sizeof(double);
+    if (t_lo < o_hi && o_lo < t_hi) return na_fail(FGD_ERR_ALIAS, "cd_sumsq overlaps theta");
+  }
   int prev = -1;
   if (cudaGetDevice(&prev) != cudaSuccess) return na_fail(FGD_ERR_CUDA, "cudaGetDevice failed");
   if (prev != device && cudaSetDevice(device) != cudaSuccess)
