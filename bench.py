@@ -83,6 +83,9 @@ def parse_args():
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
                     help="instead of the round: time the JS functional-disagreement metric on synthetic logits")
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="repeat the block of --steps rounds until the timed region lasts at least this long (0: exactly --steps rounds)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table the default run appends")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -236,6 +239,188 @@ def aggregate(dist, elapsed_ms: float, units: int, device=None):
 
 
 # ---------------------------------------------------------------------- our arm
+class RoundState:
+    """Tensors, driver and per-round launch logic of one configuration."""
+
+    def __init__(self, torch, fgd, gen, inputs_gpu, OuterRound, cfg, dev, local_rank, flags, log_rounds, seed=0):
+        self.torch, self.fgd, self.cfg, self.flags, self.seed = torch, fgd, cfg, flags, seed
+        K, P = cfg["K"], cfg["P"]
+        self.K, self.P = K, P
+        self.sig = (gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1]
+                    else np.full(K, cfg["sig"][0], np.float32))
+        self.dense_W = gen.sinkhorn_W(seed, K) if "dense" in (cfg["mix1"][0], cfg["mix2"][0]) else None
+        self.theta = torch.empty((K, P), dtype=torch.float32, device=dev)
+        self.local = torch.empty_like(self.theta)
+        self.mom = torch.zeros_like(self.theta)
+        inputs_gpu.theta0(self.theta, seed)
+        inputs_gpu.local_steps(self.local, self.theta, self.sig, seed, 0)
+        self.drv = OuterRound(K, P, device=local_rank)
+        self.cd_log = torch.zeros((log_rounds, K), dtype=torch.float64, device=dev)
+        self.main = torch.cuda.current_stream(dev)
+        self.ranges = None
+        if flags.subset_frac > 0.0:      # three blocks (embeddings, LM head, first layers), 4-column bounds
+            f = flags.subset_frac
+            q = lambda t: int(t * P) // 4 * 4
+            self.ranges = [(0, q(0.4 * f)), (q(0.5), q(0.5 + 0.3 * f)), (q(1.0 - 0.3 * f), P)]
+
+    def mix(self, which, rnd):
+        return mix_desc(self.fgd, self.cfg[which], self.cfg, rnd, self.seed, 1 if which == "mix1" else 2, self.dense_W)
+
+    def one_round(self, r, ev_pair=None):
+        """Host mix build, side-stream Mix1, fused step in place.  ev_pair brackets the step kernel alone."""
+        fl, drv, main = self.flags, self.drv, self.main
+        m1, m2 = self.mix("mix1", r), self.mix("mix2", r)
+        drv.cd_sumsq = self.cd_log[r % self.cd_log.shape[0]]
+        if fl.fuse_mix1:
+            if ev_pair is not None:
+                ev_pair[0].record(main)
+            drv.step(m2, self.local, self.theta, self.mom, self.theta, 0.7, 0.9, mix1_fused=m1, mix2_ranges=self.ranges,
+                     average_momentum=fl.average_momentum)
+            if ev_pair is not None:
+                ev_pair[1].record(main)
+            return
+        if not (fl.chain_mix1 and drv._pending is not None):
+            drv.launch_mix1(m1, self.theta)
+        if ev_pair is not None:
+            main.wait_event(drv._pending[0])     # keep the Mix1 wait out of the kernel's event pair
+            ev_pair[0].record(main)
+        drv.step(m2, self.local, self.theta, self.mom, self.theta, 0.7, 0.9, mix2_ranges=self.ranges,
+                 average_momentum=fl.average_momentum, emit_next_mix1=fl.chain_mix1)
+        if ev_pair is not None:
+            ev_pair[1].record(main)
+
+    def free(self):
+        self.theta = self.local = self.mom = self.cd_log = None
+        self.drv.close()
+        self.drv = None
+        self.torch.cuda.empty_cache()
+
+
+class Flags:
+    def __init__(self, subset_frac=0.0, average_momentum=False, chain_mix1=False, fuse_mix1=False, graph=False):
+        self.subset_frac, self.average_momentum = subset_frac, average_momentum
+        self.chain_mix1, self.fuse_mix1, self.graph = chain_mix1, fuse_mix1, graph
+
+
+MAX_TIMED_ROUNDS = 4000     # bound on the rounds (and event pairs) of one timed region
+
+
+def time_rounds(torch, st, steps, warmup, min_seconds=0.0, graph=None, barrier=None, make_sampler=None):
+    """`warmup` untimed rounds, then the timed region: the block of `steps` rounds, repeated as often
+    as it takes to fill `min_seconds` (so that the clock sampler sees the load), bracketed by
+    synchronisation on both sides; CUDA events on the launching stream around the region and around
+    every fused-step launch.  Returns the elapsed ms, the per-launch kernel ms, rounds timed, launches."""
+    main = st.main
+    probe = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+    for r in range(warmup):
+        if r == warmup - 1:
+            probe[0].record(main)
+        if graph is not None:
+            graph.replay()
+        else:
+            st.one_round(r)
+        if r == warmup - 1:
+            probe[1].record(main)
+    torch.cuda.synchronize()
+    est_ms = max(probe[0].elapsed_time(probe[1]), 1e-3)
+    repeats = 1
+    if min_seconds > 0.0:
+        repeats = max(1, int(np.ceil(min_seconds * 1e3 / (est_ms * steps))))
+        repeats = min(repeats, max(1, MAX_TIMED_ROUNDS // steps))
+    total = steps * repeats
+    if barrier is not None:
+        barrier()
+    torch.cuda.synchronize()
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(total)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = st.drv.ctx.launch_count
+    sampler = make_sampler() if make_sampler is not None else None     # clocks DURING the timed region only
+    t_begin.record(main)
+    for i in range(total):
+        if graph is not None:
+            pairs[i][0].record(main)
+            graph.replay()
+            pairs[i][1].record(main)
+        else:
+            st.one_round(warmup + i, pairs[i])
+    t_end.record(main)
+    torch.cuda.synchronize()
+    launches = st.drv.ctx.launch_count - launches0 if graph is None else 2 * total   # Mix1 kernel and fused step per replay
+    clocks = sampler.stop() if sampler is not None else None
+    return {"elapsed_ms": t_begin.elapsed_time(t_end), "kernel_ms": [a.elapsed_time(b) for a, b in pairs],
+            "rounds": total, "repeats": repeats, "launches": int(launches), "last_round": warmup + total - 1,
+            "clocks": clocks}
+
+
+def roofline_of(cfg, cfg_id, K, P, kern_times, fuse_mix1, peak, peak_kind, traffic_ok=True):
+    x_vec = cfg["mix1"][0] == "mean"
+    step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
+    mix1_bytes = (4 * K * P + 4 * P) if x_vec else 8 * K * P
+    if fuse_mix1:
+        step_bytes, mix1_bytes = 20 * K * P, 0
+    kern_ms = statistics.mean(kern_times)
+    achieved = step_bytes / (kern_ms * 1e-3) / 1e9
+    tr = (NCU_TRAFFIC_FUSED_MIX1 if fuse_mix1 else NCU_TRAFFIC_BYTES_PER_WORKER_PARAM).get(cfg_id) if traffic_ok else None
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": None if tr is None else tr * K * P,
+            "kernel": "outer_step_dense_tc_kernel" if K == 64 else "outer_step_tma_kernel",
+            "kernel_ms": kern_ms, "kernel_ms_median": statistics.median(kern_times),
+            "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
+            "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
+            "frac_of_nominal_8000": achieved / 8000.0}
+    return roof, step_bytes, mix1_bytes
+
+
+def consensus_trajectory(torch, fgd, inputs_gpu, st, rounds):
+    """The configuration's own rounds from its initial state with a fresh drift every round (untimed):
+    the consensus distance (Sec. 4.4 definition) after each.  Restores nothing: call it last."""
+    inputs_gpu.theta0(st.theta, st.seed)
+    st.mom.zero_()
+    st.drv._pending = None
+    out = []
+    for r in range(rounds):
+        if not st.flags.fuse_mix1:
+            st.drv.launch_mix1(st.mix("mix1", r), st.theta)
+        inputs_gpu.local_steps(st.local, st.theta, st.sig, st.seed, r)
+        st.drv.cd_sumsq = st.cd_log[r % st.cd_log.shape[0]]
+        st.drv.step(st.mix("mix2", r), st.local, st.theta, st.mom, st.theta, 0.7, 0.9,
+                    mix1_fused=st.mix("mix1", r) if st.flags.fuse_mix1 else None)
+        torch.cuda.synchronize()
+        out.append(fgd.fgd_cd_finalize(st.drv.cd_sumsq.cpu().numpy())[0])
+    return out
+
+
+CONFIG_ROUNDS = {1: 1, 2: 10, 3: 10, 4: 20, 5: 5, 6: 3}     # rounds each configuration asks for
+
+
+def extra_configs(torch, fgd, gen, inputs_gpu, OuterRound, dev, local_rank, peak, peak_kind, rounds=10):
+    """Configurations 1, 2, 4 (factored and with Mix1 fused) and 5 at full size, `rounds` timed
+    rounds each after 3 warm-up rounds: the fused-step kernel's time and roofline figures."""
+    out = {}
+    for key, cfg_id, fuse in (("1", 1, False), ("2", 2, False), ("4", 4, False), ("4_fused", 4, True), ("5", 5, False)):
+        cfg = CONFIGS[cfg_id]
+        st = RoundState(torch, fgd, gen, inputs_gpu, OuterRound, cfg, dev, local_rank, Flags(fuse_mix1=fuse), 64)
+        n = 200 if cfg_id == 1 else rounds
+        t = time_rounds(torch, st, n, 3)
+        roof, step_bytes, mix1_bytes = roofline_of(cfg, cfg_id, st.K, st.P, t["kernel_ms"], fuse, peak, peak_kind)
+        ms_round = t["elapsed_ms"] / t["rounds"]
+        entry = {"workload": cfg["name"] + (" [Mix1 fused into the step kernel]" if fuse else ""),
+                 "kernel": roof["kernel"],
+                 "kernel_ms": {"mean": roof["kernel_ms"], "median": roof["kernel_ms_median"], "min": roof["kernel_ms_min"],
+                               "max": roof["kernel_ms_max"]},
+                 "algorithmic_bytes": step_bytes, "achieved": roof["achieved"], "frac": roof["frac"],
+                 "frac_of_nominal_8000": roof["frac_of_nominal_8000"], "traffic": roof["traffic"],
+                 "ms_per_round": ms_round, "rounds_timed": t["rounds"], "gpu_launches": t["launches"],
+                 "worker_params_per_s": st.K * st.P / (ms_round * 1e-3)}
+        if cfg_id == 1:
+            entry["note"] = "working set fits in L2: a latency configuration, achieved/frac are not HBM figures"
+            entry["latency"] = latency_leg(torch, fgd, st.drv, cfg, st.theta, st.local, st.mom, st.seed, st.dense_W, dev)
+        out[key] = entry
+        st.free()
+        del st
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -268,134 +453,68 @@ def run_ours(args):
         cfg["name"] += f" [REDUCED to P={args.cols} for profiling: not a benchmark number]"
     K, P, seed = cfg["K"], cfg["P"], 0
     steps, warmup = args.steps, max(args.warmup, 3)
-    sig = gen.drift_sigmas(seed, K, *cfg["sig"]) if cfg["sig"][0] != cfg["sig"][1] else np.full(K, cfg["sig"][0], np.float32)
-    dense_W = gen.sinkhorn_W(seed, K) if "dense" in (cfg["mix1"][0], cfg["mix2"][0]) else None
-
-    theta = torch.empty((K, P), dtype=torch.float32, device=dev)
-    local = torch.empty_like(theta)
-    mom = torch.zeros_like(theta)
-    inputs_gpu.theta0(theta, seed)
-    inputs_gpu.local_steps(local, theta, sig, seed, 0)
-    drv = OuterRound(K, P, device=local_rank)
-    cd_log = torch.zeros((warmup + steps + 8, K), dtype=torch.float64, device=dev)
-    main = torch.cuda.current_stream(dev)
-
-    ranges = None
-    if args.subset_frac > 0.0:      # three blocks (embeddings, LM head, first layers), 4-column bounds
-        f = args.subset_frac
-        q = lambda t: int(t * P) // 4 * 4
-        ranges = [(0, q(0.4 * f)), (q(0.5), q(0.5 + 0.3 * f)), (q(1.0 - 0.3 * f), P)]
-        cfg["name"] += f" [variant: Mix2 on {sum(b - a for a, b in ranges) / P:.0%} of the columns]"
+    flags = Flags(args.subset_frac, args.average_momentum, args.chain_mix1, args.fuse_mix1, args.graph)
+    if args.fuse_mix1 and (args.chain_mix1 or args.graph or cfg["mix1"][0] == "dense"):
+        raise SystemExit("--fuse-mix1 excludes --chain-mix1 / --graph and needs a mean or sparse Mix1")
+    st = RoundState(torch, fgd, gen, inputs_gpu, OuterRound, cfg, dev, local_rank, flags, 64, seed)
+    drv, theta, local, mom, dense_W, sig = st.drv, st.theta, st.local, st.mom, st.dense_W, st.sig
+    if st.ranges is not None:
+        cfg["name"] += f" [variant: Mix2 on {sum(b - a for a, b in st.ranges) / P:.0%} of the columns]"
     if args.average_momentum:
         cfg["name"] += " [variant: momentum averaged (GlobalM1S)]"
     if args.chain_mix1:
         cfg["name"] += " [variant: Mix1 (mean) of round r+1 emitted by the fused step of round r]"
     if args.fuse_mix1:
-        if args.chain_mix1 or args.graph or cfg["mix1"][0] == "dense":
-            raise SystemExit("--fuse-mix1 excludes --chain-mix1 / --graph and needs a mean or sparse Mix1")
         cfg["name"] += " [variant: Mix1 fused into the step kernel]"
-
-    def one_round(r, ev_pair=None):
-        m1 = mix_desc(fgd, cfg["mix1"], cfg, r, seed, 1, dense_W)
-        m2 = mix_desc(fgd, cfg["mix2"], cfg, r, seed, 2, dense_W)
-        drv.cd_sumsq = cd_log[r]
-        if args.fuse_mix1:
-            if ev_pair is not None:
-                ev_pair[0].record(main)
-            drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix1_fused=m1, mix2_ranges=ranges,
-                     average_momentum=args.average_momentum)
-            if ev_pair is not None:
-                ev_pair[1].record(main)
-            return
-        if not (args.chain_mix1 and drv._pending is not None):
-            drv.launch_mix1(m1, theta)
-        if ev_pair is not None:
-            main.wait_event(drv._pending[0])     # keep the Mix1 wait out of the kernel's event pair
-            ev_pair[0].record(main)
-        drv.step(m2, local, theta, mom, theta, 0.7, 0.9, mix2_ranges=ranges, average_momentum=args.average_momentum,
-                 emit_next_mix1=args.chain_mix1)
-        if ev_pair is not None:
-            ev_pair[1].record(main)
 
     if args.kernels:
         if rank == 0:
             print(json.dumps(kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, measured_peak())), flush=True)
         return
 
-    for r in range(warmup):
-        one_round(r)
-    torch.cuda.synchronize()
     graph = None
     if args.graph:      # the whole round as ONE graph launch (static topologies only: descriptors are frozen in)
         if cfg["p_fail"] > 0.0 or "xor" in (cfg["mix1"][0], cfg["mix2"][0]) or args.chain_mix1:
             raise SystemExit("--graph needs the same Mix1 / Mix2 every round (configs 1, 3, 5)")
-        drv.cd_sumsq = cd_log[warmup]
-        graph = drv.capture(lambda: (drv.launch_mix1(mix_desc(fgd, cfg["mix1"], cfg, 0, seed, 1, dense_W), theta),
-                                     drv.step(mix_desc(fgd, cfg["mix2"], cfg, 0, seed, 2, dense_W), local, theta, mom, theta,
-                                              0.7, 0.9, mix2_ranges=ranges, average_momentum=args.average_momentum)))
+        for r in range(2):
+            st.one_round(r)         # eager calls size the launches and create the Mix1 buffer
+        torch.cuda.synchronize()
+        drv.cd_sumsq = st.cd_log[0]
+        graph = drv.capture(lambda: (drv.launch_mix1(st.mix("mix1", 0), theta),
+                                     drv.step(st.mix("mix2", 0), local, theta, mom, theta,
+                                              0.7, 0.9, mix2_ranges=st.ranges, average_momentum=args.average_momentum)))
         cfg["name"] += " [whole round replayed from one CUDA graph]"
+
+    t = time_rounds(torch, st, steps, warmup, min_seconds=args.min_seconds, graph=graph,
+                    barrier=dist.barrier if world > 1 else None,
+                    make_sampler=(lambda: ClockSampler(local_rank)) if rank == 0 else None)
+    clocks = t["clocks"]
     if world > 1:
         dist.barrier()
-    torch.cuda.synchronize()
+    elapsed_ms, units = aggregate(dist if world > 1 else None, t["elapsed_ms"], K * P, dev)
+    kern_times = t["kernel_ms"]
 
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    launches0 = drv.ctx.launch_count
-    t_begin.record(main)
-    for i in range(steps):
-        if graph is not None:
-            pairs[i][0].record(main)
-            graph.replay()
-            pairs[i][1].record(main)
-        else:
-            one_round(warmup + i, pairs[i])
-    t_end.record(main)
-    torch.cuda.synchronize()
-    launches = drv.ctx.launch_count - launches0 if graph is None else 2 * steps   # Mix1 kernel and fused step per replay
-    elapsed_ms = t_begin.elapsed_time(t_end)
-    clocks = sampler.stop() if sampler else None
-    if world > 1:
-        dist.barrier()
-    elapsed_ms, units = aggregate(dist if world > 1 else None, elapsed_ms, K * P, dev)
-    kern_times = [a.elapsed_time(b) for a, b in pairs]
-    kern_ms = statistics.mean(kern_times)
-
-    ms_per_step = elapsed_ms / steps
+    ms_per_step = elapsed_ms / t["rounds"]
     value = units / (ms_per_step * 1e-3)
-    x_vec = cfg["mix1"][0] == "mean"
-    step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
-    mix1_bytes = (4 * K * P + 4 * P) if x_vec else 8 * K * P
-    if args.fuse_mix1:
-        step_bytes, mix1_bytes = 20 * K * P, 0
     peak, peak_kind = measured_peak()
-    achieved = step_bytes / (kern_ms * 1e-3) / 1e9
-    tr = (NCU_TRAFFIC_FUSED_MIX1 if args.fuse_mix1 else NCU_TRAFFIC_BYTES_PER_WORKER_PARAM).get(args.config)
-    if args.subset_frac > 0.0 or args.average_momentum or args.chain_mix1 or args.graph:
-        tr = None                   # variants were not captured
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None if tr is None else tr * K * P,
-                "kernel": "outer_step_dense_tc_kernel" if K == 64 else "outer_step_tma_kernel",
-                "kernel_ms": kern_ms, "kernel_ms_median": statistics.median(kern_times),
-                "kernel_ms_min": min(kern_times), "kernel_ms_max": max(kern_times),
-                "algorithmic_bytes": step_bytes, "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8000": achieved / 8000.0}
-
+    variant = args.subset_frac > 0.0 or args.average_momentum or args.chain_mix1 or args.graph   # not captured with ncu
+    roofline, step_bytes, mix1_bytes = roofline_of(cfg, args.config, K, P, kern_times, args.fuse_mix1, peak, peak_kind,
+                                                   traffic_ok=not variant)
     if graph is not None:
         roofline["note"] = "graph variant: the event pair spans the whole replay (Mix1 kernel included), so achieved understates the step kernel"
-    # consensus distance of the last round (both of the paper's definitions)
-    cd_norm, cd_sq = fgd.fgd_cd_finalize(cd_log[warmup + steps - 1 if graph is None else warmup].cpu().numpy())
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": cfg["name"], "K": K, "P": P, "rounds_timed": steps,
+            "config": {"workload": cfg["name"], "K": K, "P": P, "rounds_timed": t["rounds"],
+                       "timed_region": (f"the block of {steps} rounds repeated {t['repeats']} time(s) back to back "
+                                        f"({t['rounds']} rounds, {elapsed_ms / 1e3:.2f} s) so that the clock samples cover it; "
+                                        "ms_per_step is the mean over all of them"),
                        "l2": (f"inputs {(3 * K * P * 4) / 1e9:.1f} GB per round, larger than the 126 MB L2"
                               if 3 * K * P * 4 > 4 * 126e6 else "working set fits in L2: latency config, not an HBM number"),
                        "replicas": world, "step": "host mix build + side-stream Mix1 + fused outer step with consensus sums"},
             "hbm_gbs_whole_step": (step_bytes + mix1_bytes) / (ms_per_step * 1e-3) / 1e9,
-            "roofline": roofline, "gpu_launches": int(launches), "clocks": clocks,
-            "consensus": {"cd_norm": cd_norm, "cd_sq": cd_sq}}
+            "roofline": roofline, "gpu_launches": t["launches"], "clocks": clocks}
 
     if rank == 0:
         # context: the same STREAM-style copy the pool's peak was measured with, on THIS box, now
@@ -408,9 +527,18 @@ def run_ours(args):
         line["e2e"] = None          # a pinned host copy of theta_local would take more host memory than is safe to assume
         line["config"]["e2e_note"] = "skipped: theta_local is %.0f GB, too large to pin on the host" % (K * P * 4 / 1e9)
     elif not args.no_e2e:
-        line["e2e"] = e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, cd_log, seed, dense_W, world, dev)
+        line["e2e"] = e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, st.cd_log, seed, dense_W, world, dev)
+    if rank == 0 and graph is None and not args.chain_mix1:
+        n = CONFIG_ROUNDS[args.config]
+        line["consensus"] = {"cd_norm_per_round": consensus_trajectory(torch, fgd, inputs_gpu, st, n), "rounds": n,
+                             "note": "separate untimed run of the configuration's own rounds from its initial state, fresh "
+                                     "drift every round (the timed rounds reuse one theta_local: bandwidth only)"}
+    del drv, theta, local, mom
+    st.free()
+    del st
+    if rank == 0 and world == 1 and args.config == 3 and not args.cols and not args.no_configs and not variant and not args.fuse_mix1:
+        line["configs"] = extra_configs(torch, fgd, gen, inputs_gpu, OuterRound, dev, local_rank, peak, peak_kind)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del theta, local, mom
         line["cpu_baseline"] = oracle_leg(cfg, 4, 1)[0]
         line["cpu_baseline"]["value_1thread"] = oracle_leg(cfg, 1, 0, sample_cols=1 << 19, threads=1)[0]["value"]
     if rank == 0:

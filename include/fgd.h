@@ -20,6 +20,7 @@
  * convention, row m of W = the weights worker m applies.
  *
  * Conventions for every function.
+ *  - Every entry point that launches work is wrapped in an NVTX range carrying its own name.
  *  - Returns FGD_OK (0) or a negative fgd_status.  Never throws, aborts, exits or prints.
  *    fgd_last_error() gives a human-readable reason for the last failure on that context.
  *  - Pointers named theta_*, momentum, g, in, out, x, cd_sumsq are DEVICE pointers on the
@@ -99,6 +100,18 @@ int fgd_set_path(fgd_ctx* ctx, int path);
 int fgd_device_status(fgd_ctx* ctx, void* stream);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t fgd_launch_count(const fgd_ctx* ctx);
+/* Test hooks for the bounded device-side waits (no counterpart in the paper, whose failure model
+ * -- missed exchanges, Sec. 1 / Sec. 5.2 -- is pure data: edge masks).  They let a test make a
+ * wait of the pipelined kernels run out WITHOUT faulting or hanging the GPU, to check that the
+ * kernel then records FGD_ERR_TIMEOUT, waits for its own copies, releases its tensor memory and
+ * returns, and that the context stays usable:
+ *   FGD_DEBUG_SPIN_LIMIT  polls after which a device-side wait gives up (0 = the default, 2^24);
+ *   FGD_DEBUG_SKIP_TILE   every CTA of the TMA-pipelined kernels (fused step, tensor-core step,
+ *                         tensor-core mix) announces but never issues the loads of its value-th
+ *                         tile (0-based), so the wait for that tile runs out; -1 = off (default).
+ * Both stay set until changed.  Not for production use. */
+typedef enum { FGD_DEBUG_SPIN_LIMIT = 1, FGD_DEBUG_SKIP_TILE = 2 } fgd_debug_key;
+int fgd_debug_set(fgd_ctx* ctx, int key, int64_t value);
 
 /* ---- mixing operators (Sec. 3 "Gossip-based Mixing"; App. A table of (Mix1, Mix2)) ---- */
 typedef enum {

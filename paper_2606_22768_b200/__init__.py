@@ -65,6 +65,7 @@ def _load():
         "fgd_launch_count": (i64, [vp]),
         "fgd_set_path": (i32, [vp, i32]),
         "fgd_device_status": (i32, [vp, vp]),
+        "fgd_debug_set": (i32, [vp, i32, i64]),
         "fgd_outer_grad": (i32, [vp, vp, vp, vp, vp]),
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
@@ -274,6 +275,14 @@ class Context:
 
 def fgd_set_path(ctx: Context, path: int) -> None:
     ctx._check(_lib.fgd_set_path(ctx._h, int(path)))
+
+
+FGD_DEBUG_SPIN_LIMIT, FGD_DEBUG_SKIP_TILE = 1, 2
+
+
+def fgd_debug_set(ctx: Context, key: int, value: int) -> None:
+    """Test hooks of the bounded device-side waits (see ``include/fgd.h``)."""
+    ctx._check(_lib.fgd_debug_set(ctx._h, int(key), int(value)))
 
 
 def fgd_device_status(ctx: Context, stream=None) -> None:

@@ -8,6 +8,7 @@
 
 #include "fgd_ctx.h"
 #include "fgd_kernels.cuh"
+#include "fgd_nvtx.h"
 #include "fgd_step_tma.h"
 
 using namespace fgd;
@@ -15,6 +16,7 @@ using namespace fgd;
 extern "C" {
 
 int fgd_create(fgd_ctx** out, int device, int K, int64_t P, int64_t ld) {
+  FGD_NVTX_RANGE("fgd_create");
   if (!out) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_create: out is NULL");
   *out = nullptr;
   if (K < 1 || K > FGD_MAX_K) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_create: K=%d out of range [1, %d]", K, FGD_MAX_K);
@@ -81,6 +83,7 @@ int fgd_set_path(fgd_ctx* c, int path) {
 }
 
 int fgd_device_status(fgd_ctx* c, void* stream) {
+  FGD_NVTX_RANGE("fgd_device_status");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_device_status: ctx is NULL");
   DeviceGuard guard(c->device);
   if (!guard.ok) return fail(c, FGD_ERR_CUDA, "cannot select device %d", c->device);
@@ -96,7 +99,24 @@ int fgd_device_status(fgd_ctx* c, void* stream) {
 }
 int64_t fgd_launch_count(const fgd_ctx* c) { return c ? c->launches : 0; }
 
+int fgd_debug_set(fgd_ctx* c, int key, int64_t value) {
+  if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_debug_set: ctx is NULL");
+  switch (key) {
+    case FGD_DEBUG_SPIN_LIMIT:
+      if (value < 0 || value > (int64_t)0xffffffffu) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: spin limit %lld out of range", (long long)value);
+      c->dbg_spin_limit = (uint32_t)value;
+      return FGD_OK;
+    case FGD_DEBUG_SKIP_TILE:
+      if (value < -1 || value > 0x7fffffff) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: tile index %lld out of range", (long long)value);
+      c->dbg_skip_tile = (int)value;
+      return FGD_OK;
+    default:
+      return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: unknown key %d", key);
+  }
+}
+
 int fgd_outer_grad(fgd_ctx* c, const float* theta_prev, const float* theta_local, float* g, void* stream) {
+  FGD_NVTX_RANGE("fgd_outer_grad");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_outer_grad: ctx is NULL");
   if (!theta_prev || !theta_local || !g) return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_grad: NULL tensor");
   const Range rg = mat_range(g, c->K, c->P, c->ld);
@@ -117,6 +137,7 @@ int fgd_outer_grad(fgd_ctx* c, const float* theta_prev, const float* theta_local
 }
 
 int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, int out_is_vector, void* stream) {
+  FGD_NVTX_RANGE("fgd_mix");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_mix: ctx is NULL");
   if (!in || !out) return fail(c, FGD_ERR_INVALID_ARG, "fgd_mix: NULL tensor");
   if (int rc = validate_desc(desc, c->K, c->err, sizeof(c->err))) return rc;
@@ -215,6 +236,7 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
                       int x_is_vector, const float* theta_local, const float* theta_prev, float* momentum,
                       float* theta_new, double lr, double mu, double* cd_sumsq, const fgd_step_options* opts,
                       void* stream) {
+  FGD_NVTX_RANGE("fgd_outer_step_ex");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_outer_step: ctx is NULL");
   if (!theta_local || !theta_prev || !momentum || !theta_new)
     return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_step: NULL tensor");
@@ -369,6 +391,7 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
 }
 
 int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, void* stream) {
+  FGD_NVTX_RANGE("fgd_consensus_distance");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_consensus_distance: ctx is NULL");
   if (!theta || !cd_sumsq) return fail(c, FGD_ERR_INVALID_ARG, "fgd_consensus_distance: NULL pointer");
   if (overlap(vec_range(cd_sumsq, c->K, sizeof(double)), mat_range(theta, c->K, c->P, c->ld)))

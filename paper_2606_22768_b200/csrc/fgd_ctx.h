@@ -34,6 +34,8 @@ struct fgd_ctx {
   int max_smem_optin = 0;
   void* encode_tiled = nullptr;  // cuTensorMapEncodeTiled, resolved through the runtime
   int64_t launches = 0;
+  uint32_t dbg_spin_limit = 0;   // fgd_debug_set: polls before a device-side wait gives up (0 = the default)
+  int dbg_skip_tile = -1;        // fgd_debug_set: tile whose loads the pipelined kernels withhold (-1 = none)
   char err[256] = "";
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
   // fgd_outer_step_from_host only (created by its first call): copy stream, one event per column

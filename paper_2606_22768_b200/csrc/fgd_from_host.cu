@@ -4,6 +4,7 @@
 
 #include "../../include/fgd.h"
 #include "fgd_ctx.h"
+#include "fgd_nvtx.h"
 
 namespace {
 
@@ -61,6 +62,7 @@ extern "C" int fgd_outer_step_from_host(fgd_ctx* c, const fgd_mix_desc* mix2, co
                                         float* theta_local_dev, const float* theta_prev, float* momentum,
                                         float* theta_new, double lr, double mu, double* cd_sumsq_host,
                                         int n_chunks, void* stream) {
+  FGD_NVTX_RANGE("fgd_outer_step_from_host");
   if (!c) return fail(nullptr, FGD_ERR_INVALID_ARG, "fgd_outer_step_from_host: ctx is NULL");
   if (!theta_local_host || !theta_local_dev || !theta_prev || !momentum || !theta_new)
     return fail(c, FGD_ERR_INVALID_ARG, "fgd_outer_step_from_host: NULL tensor");

@@ -25,6 +25,8 @@ struct TcMixArgs {
   int64_t P, ld;
   int K;
   int* status;
+  uint32_t spin_limit;   // polls before a bounded wait gives up
+  int skip_tile;         // test hook, see TmaStepArgs
 };
 
 template <int KP, bool FULL>
@@ -84,18 +86,20 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
       for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
         const int s = (int)(i % STAGES);
         const uint32_t use = (uint32_t)(i / STAGES);
-        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1);
+        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1, a.spin_limit);
         if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
         const uint32_t full = smem_u32(&bars[s]);
         mbar_expect_tx(full, BOX);
+        if (i == a.skip_tile) continue;            // test hook: this load never arrives
         tma_load_2d(smem_u32(base + (size_t)s * 2 * BOX), &tm_in, (int)(tile * T), 0, full, policy);
       }
       if (!ok) {
         *(volatile int*)&abort_flag = 1;
         atomicExch(a.status, FGD_ERR_TIMEOUT);
-        for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
-          mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1);
       }
+      // never exit under a copy in flight: bounded wait for the last use of every stage
+      for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
+        if (j != a.skip_tile) mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1, a.spin_limit);
     }
   } else {
     // ===================================================== consumers: thread (c, h) = column c, workers [H h, H h + H)
@@ -113,7 +117,7 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
       float* A = reinterpret_cast<float*>(stage);          // in box -> hi operand
       unsigned char* L = stage + BOX;                      // lo operand
       float v[H];
-      if (mbar_wait(smem_u32(&bars[s]), use & 1)) {
+      if (mbar_wait(smem_u32(&bars[s]), use & 1, a.spin_limit)) {
 #pragma unroll
         for (int n = 0; n < H; ++n) v[n] = A[(r0 + n) * T + c];
       } else {
@@ -153,7 +157,7 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
         }
         umma_commit(mma_bar);
       }
-      if (!mbar_wait(mma_bar, (uint32_t)i & 1)) {
+      if (!mbar_wait(mma_bar, (uint32_t)i & 1, a.spin_limit)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(a.status, FGD_ERR_TIMEOUT);
       }

@@ -18,6 +18,7 @@
 #include <mutex>
 
 #include "fgd_kernels.cuh"
+#include "fgd_nvtx.h"
 
 using namespace fgd;
 
@@ -86,6 +87,7 @@ int launch_consensus(const float* theta, double* scratch, int K, int64_t P, int6
 
 extern "C" int fgd_consensus_distance_noalloc(int device, int K, int64_t P, int64_t ld, const float* theta,
                                               double* cd_sumsq, void* stream) {
+  FGD_NVTX_RANGE("fgd_consensus_distance_noalloc");
   if (device < 0 || device >= kMaxDevices) return na_fail(FGD_ERR_INVALID_ARG, "device %d out of range", device);
   if (K < 1 || K > FGD_MAX_K)
     return na_fail(FGD_ERR_INVALID_ARG,

@@ -241,10 +241,11 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
         const int s = (int)(i % STAGES);
         const uint32_t use = (uint32_t)(i / STAGES);
-        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1);
+        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1, ta.spin_limit);
         if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
         const uint32_t full = smem_u32(&bars[s]);
         mbar_expect_tx(full, 3 * kTcBox);
+        if (i == ta.skip_tile) continue;           // test hook: these loads never arrive
         const uint32_t dst = smem_u32(base + (size_t)s * 3 * kTcBox);
         const int c0 = (int)(tile * T);
         tma_load_2d(dst, &tm_prev, c0, 0, full, policy);
@@ -256,9 +257,10 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       if (!ok) {
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
-        for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
-          mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1);
       }
+      // never exit under a copy in flight: bounded wait for the last use of every stage
+      for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
+        if (j != ta.skip_tile) mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1, ta.spin_limit);
     }
   } else {
     // ===================================================== consumers
@@ -302,7 +304,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
       // ---- phase 1: g of this thread's workers in registers
       float g[H];
       float tsum = 0.f;
-      const bool got = mbar_wait(smem_u32(&bars[s]), use & 1);
+      const bool got = mbar_wait(smem_u32(&bars[s]), use & 1, ta.spin_limit);
       if (got) {
 #pragma unroll
         for (int n = 0; n < H; ++n) {
@@ -376,7 +378,7 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
         for (int m = 0; m < H; ++m) v[m] = vs;
       }
       if (need_tsum) xv = tsum * invK;
-      if (!mbar_wait(mma_bar, (uint32_t)(i / NG) & 1)) {
+      if (!mbar_wait(mma_bar, (uint32_t)(i / NG) & 1, ta.spin_limit)) {
         *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
       }

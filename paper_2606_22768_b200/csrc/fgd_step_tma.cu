@@ -73,6 +73,8 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const StepArgs& a, const DenseMix& d2, 
   ta.s = a;
   ta.status = c->status;
   ta.n_tensors = (a.xsrc == XSRC_MATRIX && aligned16(a.x)) ? 4 : 3;
+  ta.spin_limit = c->dbg_spin_limit ? c->dbg_spin_limit : kSpinLimit;
+  ta.skip_tile = c->dbg_skip_tile;
   int rc = FGD_OK;
   switch (tc_padded_k(c->K)) {
     case 32: ta.stages = TcShape<32>::kStages; rc = launch_tc<32>(c, ta, d2, g1, st, grid_out); break;
@@ -107,7 +109,7 @@ static int launch_mix_tc(fgd_ctx* c, const TcMixArgs& a, const DenseMix& dm, cud
 }
 
 int fgd_launch_mix_dense_tc(fgd_ctx* c, const float* in, float* out, const DenseMix& dm, cudaStream_t st) {
-  const TcMixArgs a{in, out, c->P, c->ld, c->K, c->status};
+  const TcMixArgs a{in, out, c->P, c->ld, c->K, c->status, c->dbg_spin_limit ? c->dbg_spin_limit : kSpinLimit, c->dbg_skip_tile};
   int rc = FGD_OK;
   switch (tc_padded_k(c->K)) {
     case 32: rc = launch_mix_tc<32>(c, a, dm, st); break;

@@ -23,7 +23,7 @@
 
 namespace fgd {
 
-constexpr uint32_t kSpinLimit = 1u << 24;  // try_wait iterations before a wait gives up
+constexpr uint32_t kSpinLimit = 1u << 24;  // try_wait iterations before a wait gives up (the launch may pass a smaller limit)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -37,9 +37,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Bounded wait for the phase with the given parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+// Bounded wait for the phase with the given parity; false = gave up after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -70,6 +70,9 @@ struct TmaStepArgs {
   int* status;       // device status word (0 = ok)
   int n_tensors;     // 3, or 4 when x is a [K, ld] matrix
   int stages;        // pipeline depth, 2..kMaxStages
+  uint32_t spin_limit;  // polls before a bounded wait gives up (kSpinLimit unless a test shortened it)
+  int skip_tile;     // test hook: the producer announces but does not issue the loads of each CTA's
+                     // skip_tile-th tile, so that the consumers' wait runs out; -1 = off
 };
 
 // Shared-memory need of the kernel (bytes), also used by the host to size the launch.
@@ -146,13 +149,14 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
       for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
         const int s = (int)(i % STAGES);
         const uint32_t use = (uint32_t)(i / STAGES);
-        if (use > 0) ok = mbar_wait(smem_u32(&bars[kMaxStages + s]), (use - 1) & 1);
+        if (use > 0) ok = mbar_wait(smem_u32(&bars[kMaxStages + s]), (use - 1) & 1, ta.spin_limit);
         if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
         const uint32_t full = smem_u32(&bars[s]);
         const int64_t c0 = tile * T;
         const int64_t left = P - c0;                                  // > 0
         const int nbox = left >= T ? NBOX : (int)((left + BOXC - 1) / BOXC);   // boxes that touch the tensor
         mbar_expect_tx(full, (uint32_t)(box_floats * sizeof(float)) * (uint32_t)(nbox * NT));
+        if (i == ta.skip_tile) continue;                              // test hook: these loads never arrive
         const uint32_t dst = smem_u32(stages + stage_floats * s);
         for (int b = 0; b < nbox; ++b) {
           const uint32_t d = dst + (uint32_t)(box_floats * sizeof(float)) * b;
@@ -163,13 +167,14 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           if (NT == 4) tma_load_2d(d + (uint32_t)(tens_floats * 12), &tm_x, c, 0, full, policy);
         }
       }
-      if (!ok) {
-        // give up: flag it, then wait (bounded) for every copy this thread still has in flight
+      if (!ok) {   // give up: flag it
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
-        for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
-          mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1);
       }
+      // The CTA must not exit under a copy that is still in flight (the consumers may have given up
+      // early): wait, bounded, for the last use of every stage.  In a healthy run these have landed.
+      for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
+        if (j != ta.skip_tile) mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1, ta.spin_limit);
     }
   } else {
     // ===================================================== consumers
@@ -215,7 +220,8 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           for (int q = 0; q < VEC; ++q)
             if (col + q < P) xv.v[q] = a.x[col + q];
       }
-      if (!mbar_wait(smem_u32(&bars[s]), use & 1)) {
+      // (the give-up decision is taken per warp, so a warp never leaves the loop half way)
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars[s]), use & 1, ta.spin_limit))) {
         *(volatile int*)&abort_flag = 1;
         atomicExch(ta.status, FGD_ERR_TIMEOUT);
         break;

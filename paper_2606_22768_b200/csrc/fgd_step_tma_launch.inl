@@ -13,6 +13,8 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   ta.status = c->status;
   ta.n_tensors = tma_n_tensors(a, KT, dense2);
   ta.stages = sh.stages;
+  ta.spin_limit = c->dbg_spin_limit ? c->dbg_spin_limit : kSpinLimit;
+  ta.skip_tile = c->dbg_skip_tile;
   const int T = sh.consumers * sh.vec;
   const int boxc = T < 256 ? T : 256;
   CUtensorMap tp, tl, tm, tx;
