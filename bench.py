@@ -79,6 +79,7 @@ def parse_args():
                     help="variant: capture the round (Mix1 + fused step) into one CUDA graph and time its replays")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the round: the fused step across worker counts and mix kinds (4 GB per tensor)")
+    ap.add_argument("--sweep-ks", default="", help="with --sweep: comma-separated worker counts (default: the full list)")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
@@ -445,7 +446,8 @@ def run_ours(args):
         return
     if args.sweep:
         if rank == 0:
-            print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak())), flush=True)
+            ks = tuple(int(k) for k in args.sweep_ks.split(",")) if args.sweep_ks else None
+            print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak(), **({"Ks": ks} if ks else {}))), flush=True)
         return
     cfg = dict(CONFIGS[args.config])
     if args.cols:

@@ -1,9 +1,23 @@
-// Stand-alone mix out = W in for 17 <= K <= 64 on the tensor cores: the same tcgen05 3xTF32
-// contraction, operand layout and TMA / mbarrier / TMEM choreography as the fused step in
-// fgd_step_dense_tc.cuh, with one tensor per stage.  A stage holds the [KP x 128] box of `in`
-// (overwritten in place by its tf32-rounded half, the A operand "hi") and a second buffer of the
-// same size for the remainders ("lo").  Any mix is a dense matrix, so sparse mixes at these worker
-// counts are densified by the caller and take this kernel too.
+// Stand-alone mix out = W in for 17 <= K <= 64 on the tensor cores: the tcgen05 3xTF32 contraction
+// of the fused step (fgd_step_dense_tc.cuh: same W operand in shared memory, same split
+//     W v ~= W_hi v_hi + W_hi v_lo + W_lo v_hi,  fp32 accumulators in tensor memory)
+// with a data flow of its own.  A mix moves only 8 bytes per worker-parameter, so per tile the
+// contraction, the tensor-memory round trip and the barrier hand-offs weigh much more than in the
+// step; a kernel that holds its stage across them has one tile in flight per SM and is latency-bound.
+// Here nothing waits on the arithmetic:
+//   * the A operand v^T (M = 128 columns of the tile, K = workers) is read by the MMA from TENSOR
+//     MEMORY: a consumer thread reads its H values of the staged box, splits them and writes v_hi /
+//     v_lo into its own TMEM lane (lane = column) with tcgen05.st.  Shared memory is only the landing
+//     zone of the TMA boxes -- a stage goes back to the producer as soon as the consumers hold it in
+//     registers -- so the ring is deep (one 32 KB box per stage at K = 64: six stages in flight);
+//   * operand buffers and accumulator are double-buffered in TMEM and a dedicated warp issues the
+//     MMAs: the contraction of tile i runs while the consumers store the result of tile i - 1 and
+//     read tile i + 1.
+// Warps 0-7 consumers (thread (c, h): column c, workers [H h, H h + H)), warp 8 lane 0 TMA
+// producer, warp 9 lane 0 MMA issuer (warp 9 owns the tensor-memory allocation).  Any mix is a
+// dense matrix, so sparse mixes at these worker counts are densified by the caller and take this
+// kernel too.  Every wait is bounded and gives up early once the CTA's abort flag is up; the
+// producer waits for its copies, the MMA warp for its last commits, tensor memory is released.
 #ifndef FGD_MIX_DENSE_TC_CUH_
 #define FGD_MIX_DENSE_TC_CUH_
 
@@ -11,12 +25,43 @@
 
 namespace fgd {
 
+// tcgen05.mma with the A operand in tensor memory (lane = row of A, one 32-bit column per k).
+__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+
+// Bounded wait that also gives up when the CTA's abort flag is up (looked at every 32 polls).
+__device__ __forceinline__ bool mbar_wait_or_abort(uint32_t bar, uint32_t parity, uint32_t limit, const int* abort_flag) {
+  for (uint32_t it = 0; it < limit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 31u) == 31u && *(const volatile int*)abort_flag) return false;
+  }
+  return false;
+}
+
 template <int KP>
 struct TcMixShape {
   using S = TcShape<KP>;
-  static constexpr int kStages = KP <= 32 ? 4 : 3;
-  // dynamic shared memory: alignment slack + stages x (box + lo buffer) + W_hi + W_lo
-  static constexpr size_t kSmem = 128 + (size_t)kStages * 2 * S::kBox + 2 * S::kWBytes;
+  static constexpr int kCW = KP <= 32 ? 32 : 64;              // tensor-memory columns per buffer
+  static constexpr int kTmemCols = KP <= 32 ? 256 : 512;      // 2 accumulators + 2 v_hi + 2 v_lo, a power of two
+  static constexpr int kThreads = kTcConsumers + 64;          // consumers + producer warp + MMA warp
+  // as many one-box stages as fit beside W_hi and W_lo (at most 8)
+  static constexpr int kFit = (int)((227u * 1024u - 1024u - 128u - 2u * S::kWBytes) / S::kBox);
+  static constexpr int kStages = kFit > 8 ? 8 : kFit;
+  static constexpr size_t kSmem = 128 + (size_t)kStages * S::kBox + 2 * S::kWBytes;
 };
 
 struct TcMixArgs {
@@ -30,35 +75,43 @@ struct TcMixArgs {
 };
 
 template <int KP, bool FULL>
-__global__ void __launch_bounds__(kTcConsumers + 32)
+__global__ void __launch_bounds__(TcMixShape<KP>::kThreads, 1)
 mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant__ CUtensorMap tm_in) {
   using Shape = TcShape<KP>;
   constexpr int K = KP, T = kTcCols, H = Shape::kHalf, CONS = kTcConsumers, STAGES = TcMixShape<KP>::kStages;
+  constexpr int CW = TcMixShape<KP>::kCW;
   constexpr uint32_t BOX = Shape::kBox, WB = Shape::kWBytes, SBO = Shape::kSbo;
   const int KR = FULL ? K : a.K;
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];   // full[], empty[], mma
+  // full[STAGES], empty[STAGES], ready[2] (operands of buffer b stored), mma[2] (accumulator b complete)
+  __shared__ __align__(8) unsigned long long bars[2 * STAGES + 4];
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_slot;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   unsigned char* base = smem_raw + ((128u - (smem_u32(smem_raw) & 127u)) & 127u);
-  unsigned char* wb_hi = base + (size_t)STAGES * 2 * BOX;
+  unsigned char* wb_hi = base + (size_t)STAGES * BOX;
   unsigned char* wb_lo = wb_hi + WB;
-  const uint32_t mma_bar = smem_u32(&bars[2 * STAGES]);
+  const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[STAGES]);
+  const uint32_t bar_ready = smem_u32(&bars[2 * STAGES]), bar_mma = smem_u32(&bars[2 * STAGES + 2]);
+  const uint32_t spin = a.spin_limit;
   const int64_t P = a.P, ld = a.ld;
   const int64_t ntiles = (P + T - 1) / T;
+  const int64_t my_tiles = ntiles > blockIdx.x ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
   if (tid == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bars[s]), 1);
-      mbar_init(smem_u32(&bars[STAGES + s]), CONS);
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, CONS / 32);     // one arrival per consumer warp
     }
-    mbar_init(mma_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_ready + 8u * b, CONS / 32);
+      mbar_init(bar_mma + 8u * b, 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i < K * K; i += CONS + 32) {   // B operand = W^T, K-major core matrices, zero-padded
+  for (int i = tid; i < K * K; i += TcMixShape<KP>::kThreads) {   // B operand = W^T, K-major core matrices, zero-padded
     const int n = i / K, m = i % K;
     const float w = (FULL || (n < KR && m < KR)) ? mx.Wt[n * KR + m] : 0.f;
     const float hi = to_tf32(w);
@@ -66,8 +119,8 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
     *reinterpret_cast<float*>(wb_hi + off) = hi;
     *reinterpret_cast<float*>(wb_lo + off) = w - hi;
   }
-  if (warp == CONS / 32) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)Shape::kTmemCols) : "memory");
+  if (warp == CONS / 32 + 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)TcMixShape<KP>::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -77,7 +130,7 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
   const uint32_t tmem_base = tmem_base_slot;
 
   if (warp == CONS / 32) {
-    // ===================================================== producer (one elected lane)
+    // ===================================================== TMA producer (one elected lane)
     if (lane == 0) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
@@ -86,12 +139,12 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
       for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++i) {
         const int s = (int)(i % STAGES);
         const uint32_t use = (uint32_t)(i / STAGES);
-        if (use > 0) ok = mbar_wait(smem_u32(&bars[STAGES + s]), (use - 1) & 1, a.spin_limit);
+        if (use > 0) ok = mbar_wait_or_abort(bar_empty + 8u * s, (use - 1) & 1, spin, &abort_flag);
         if (!ok || *(volatile int*)&abort_flag) { ok = false; break; }
-        const uint32_t full = smem_u32(&bars[s]);
+        const uint32_t full = bar_full + 8u * s;
         mbar_expect_tx(full, BOX);
         if (i == a.skip_tile) continue;            // test hook: this load never arrives
-        tma_load_2d(smem_u32(base + (size_t)s * 2 * BOX), &tm_in, (int)(tile * T), 0, full, policy);
+        tma_load_2d(smem_u32(base + (size_t)s * BOX), &tm_in, (int)(tile * T), 0, full, policy);
       }
       if (!ok) {
         *(volatile int*)&abort_flag = 1;
@@ -99,78 +152,100 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
       }
       // never exit under a copy in flight: bounded wait for the last use of every stage
       for (int64_t j = (i > STAGES ? i - STAGES : 0); j < i; ++j)
-        if (j != a.skip_tile) mbar_wait(smem_u32(&bars[j % STAGES]), (uint32_t)(j / STAGES) & 1, a.spin_limit);
+        if (j != a.skip_tile) mbar_wait(bar_full + 8u * (uint32_t)(j % STAGES), (uint32_t)(j / STAGES) & 1, spin);
+    }
+  } else if (warp == CONS / 32 + 1) {
+    // ===================================================== MMA issuer (one elected lane)
+    if (lane == 0) {
+      // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
+      constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
+      const uint32_t b_hi = smem_u32(wb_hi), b_lo = smem_u32(wb_lo);
+      int64_t i = 0;
+      for (; i < my_tiles; ++i) {
+        const uint32_t b = (uint32_t)(i & 1);
+        if (!mbar_wait_or_abort(bar_ready + 8u * b, (uint32_t)(i >> 1) & 1, spin, &abort_flag)) {
+          *(volatile int*)&abort_flag = 1;
+          atomicExch(a.status, FGD_ERR_TIMEOUT);
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = tmem_base + b * CW;
+        const uint32_t a_hi = tmem_base + (2 + b) * CW, a_lo = tmem_base + (4 + b) * CW;
+#pragma unroll
+        for (int prod = 0; prod < 3; ++prod) {     // W_hi v_hi, W_hi v_lo, W_lo v_hi
+          const uint32_t aa = prod == 1 ? a_lo : a_hi;
+          const uint32_t bb = prod == 2 ? b_lo : b_hi;
+#pragma unroll
+          for (int ks = 0; ks < K / 8; ++ks) {
+            const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, SBO, 0u);
+            umma_tf32_ts(acc, aa + (uint32_t)ks * 8u, db, idesc, (prod | ks) ? 1u : 0u);
+          }
+        }
+        umma_commit(bar_mma + 8u * b);
+      }
+      // tensor memory must not be released under a running MMA: wait (bounded) for the last commits
+      for (int64_t j = (i > 2 ? i - 2 : 0); j < i; ++j)
+        mbar_wait(bar_mma + 8u * (uint32_t)(j & 1), (uint32_t)(j >> 1) & 1, spin);
     }
   } else {
     // ===================================================== consumers: thread (c, h) = column c, workers [H h, H h + H)
     const int c = tid & (T - 1), h = tid >> 7, r0 = h * H;
     const int hr = FULL ? H : min(max(KR - r0, 0), H);
-    const uint32_t op_row = (uint32_t)(c >> 3) * SBO + (uint32_t)(c & 7) * 16u;
-    constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
-    int64_t i = 0;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
-      const int s = (int)(i % STAGES);
-      const uint32_t use = (uint32_t)(i / STAGES);
-      const int64_t col = tile * T + c;
-      const bool live = col < P;
-      unsigned char* stage = base + (size_t)s * 2 * BOX;
-      float* A = reinterpret_cast<float*>(stage);          // in box -> hi operand
-      unsigned char* L = stage + BOX;                      // lo operand
-      float v[H];
-      if (mbar_wait(smem_u32(&bars[s]), use & 1, a.spin_limit)) {
+    const uint32_t t_acc = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0;   // + b * CW
+    const uint32_t t_hi = t_acc + 2 * CW, t_lo = t_acc + 4 * CW;
+    for (int64_t i = 0; i <= my_tiles; ++i) {
+      if (i < my_tiles) {
+        // ---------------- tile i: box -> registers -> split -> operand buffers i & 1
+        const int s = (int)(i % STAGES);
+        const uint32_t b = (uint32_t)(i & 1);
+        const float* A = reinterpret_cast<const float*>(base + (size_t)s * BOX);
+        if (!mbar_wait_or_abort(bar_full + 8u * s, (uint32_t)(i / STAGES) & 1, spin, &abort_flag)) {
+          *(volatile int*)&abort_flag = 1;
+          atomicExch(a.status, FGD_ERR_TIMEOUT);
+          break;
+        }
+        float v[H];
 #pragma unroll
         for (int n = 0; n < H; ++n) v[n] = A[(r0 + n) * T + c];
-      } else {
-        *(volatile int*)&abort_flag = 1;
-        atomicExch(a.status, FGD_ERR_TIMEOUT);
-      }
-      named_bar_sync(1, CONS);                    // every consumer has read its rows of the box
-      if (*(volatile int*)&abort_flag) break;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty + 8u * s);       // the box is in registers: refill the stage
 #pragma unroll
-      for (int n = 0; n < H; n += 4) {
-        float4 hi, lo;
-        hi.x = to_tf32(v[n]);     lo.x = v[n] - hi.x;
-        hi.y = to_tf32(v[n + 1]); lo.y = v[n + 1] - hi.y;
-        hi.z = to_tf32(v[n + 2]); lo.z = v[n + 2] - hi.z;
-        hi.w = to_tf32(v[n + 3]); lo.w = v[n + 3] - hi.w;
-        const uint32_t off = op_row + (uint32_t)((r0 + n) >> 2) * 128u;
-        *reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(A) + off) = hi;
-        *reinterpret_cast<float4*>(L + off) = lo;
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      named_bar_sync(2, CONS);                    // operands complete; last tile's TMEM reads are done too
-      if (tid == 0) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_hi = smem_u32(A), a_lo = smem_u32(L);
-        const uint32_t b_hi = smem_u32(wb_hi), b_lo = smem_u32(wb_lo);
+        for (int n = 0; n < H; n += 8) {
+          float hi[8], lo[8];
 #pragma unroll
-        for (int prod = 0; prod < 3; ++prod) {     // W_hi in_hi, W_hi in_lo, W_lo in_hi
-          const uint32_t aa = prod == 1 ? a_lo : a_hi;
-          const uint32_t bb = prod == 2 ? b_lo : b_hi;
-#pragma unroll
-          for (int ks = 0; ks < K / 8; ++ks) {
-            const uint64_t da = umma_desc(aa + (uint32_t)ks * 256u, 128u, SBO, 0u);
-            const uint64_t db = umma_desc(bb + (uint32_t)ks * 256u, 128u, SBO, 0u);
-            umma_tf32(tmem_base, da, db, idesc, (prod | ks) ? 1u : 0u);
+          for (int q = 0; q < 8; ++q) {
+            hi[q] = to_tf32(v[n + q]);
+            lo[q] = v[n + q] - hi[q];
           }
+          tmem_st_8(t_hi + b * CW + (uint32_t)n, hi);
+          tmem_st_8(t_lo + b * CW + (uint32_t)n, lo);
         }
-        umma_commit(mma_bar);
+        tmem_st_wait();
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_ready + 8u * b);
       }
-      if (!mbar_wait(mma_bar, (uint32_t)i & 1, a.spin_limit)) {
-        *(volatile int*)&abort_flag = 1;          // seen by everyone at the next tile's barrier
-        atomicExch(a.status, FGD_ERR_TIMEOUT);
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(smem_u32(&bars[STAGES + s]));   // the MMA has consumed the operands: the stage can be refilled
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float r[H];
-      tmem_ld_cols<H>(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)r0, r);
-      if (live) {
-        float* const out_col = a.out + (size_t)r0 * ld + col;
+      if (i > 0) {
+        // ---------------- tile i - 1: accumulator -> HBM
+        const int64_t j = i - 1;
+        const uint32_t b = (uint32_t)(j & 1);
+        const int64_t col = (blockIdx.x + j * (int64_t)gridDim.x) * T + c;
+        if (!mbar_wait_or_abort(bar_mma + 8u * b, (uint32_t)(j >> 1) & 1, spin, &abort_flag)) {
+          *(volatile int*)&abort_flag = 1;
+          atomicExch(a.status, FGD_ERR_TIMEOUT);
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float r[H];
+        tmem_ld_cols<H>(t_acc + b * CW, r);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");   // ordered before what this thread signals next
+        if (col < P) {
+          float* const out_col = a.out + (size_t)r0 * ld + col;
 #pragma unroll
-        for (int m = 0; m < H; ++m) {
-          if (FULL || m < hr) __stcs(out_col + (size_t)m * ld, r[m]);
+          for (int m = 0; m < H; ++m) {
+            if (FULL || m < hr) __stcs(out_col + (size_t)m * ld, r[m]);
+          }
         }
       }
     }
@@ -178,9 +253,9 @@ mix_dense_tc_kernel(const TcMixArgs a, const DenseMix mx, const __grid_constant_
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == CONS / 32) {
+  if (warp == CONS / 32 + 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Shape::kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TcMixShape<KP>::kTmemCols) : "memory");
   }
 }
 

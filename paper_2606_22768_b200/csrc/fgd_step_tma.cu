@@ -91,7 +91,7 @@ bool fgd_mix_tc_eligible(const fgd_ctx* c, const float* in, bool really_dense) {
   const int K = c->K;
   if (K > kTcMaxK || K < kTcMinK || kt_of(K) == 16 || (kt_of(K) == 32 && !really_dense)) return false;
   if (!c->encode_tiled || c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096 || !aligned16(in)) return false;
-  return (size_t)c->max_smem_optin >= TcMixShape<kTcMaxK>::kSmem + 256;
+  return (size_t)c->max_smem_optin >= TcMixShape<kTcMaxK>::kSmem + 512;
 }
 
 template <int KP>
@@ -101,8 +101,8 @@ static int launch_mix_tc(fgd_ctx* c, const TcMixArgs& a, const DenseMix& dm, cud
   const int64_t ntiles = (c->P + kTcCols - 1) / kTcCols;
   int grid = 0;
   auto launch = [&](auto kern) -> int {
-    if (int r = persistent_grid(c, kern, kTcConsumers + 32, TcMixShape<KP>::kSmem, ntiles, &grid)) return r;
-    kern<<<grid, kTcConsumers + 32, TcMixShape<KP>::kSmem, st>>>(a, dm, tin);
+    if (int r = persistent_grid(c, kern, TcMixShape<KP>::kThreads, TcMixShape<KP>::kSmem, ntiles, &grid)) return r;
+    kern<<<grid, TcMixShape<KP>::kThreads, TcMixShape<KP>::kSmem, st>>>(a, dm, tin);
     return FGD_OK;
   };
   return c->K == KP ? launch(mix_dense_tc_kernel<KP, true>) : launch(mix_dense_tc_kernel<KP, false>);
