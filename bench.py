@@ -87,6 +87,7 @@ def parse_args():
     ap.add_argument("--min-seconds", type=float, default=2.0,
                     help="repeat the block of --steps rounds until the timed region lasts at least this long (0: exactly --steps rounds)")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table the default run appends")
+    ap.add_argument("--js-positions", type=int, default=4096, help="with --js: token positions U (reduce for profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -442,7 +443,7 @@ def run_ours(args):
 
     if args.js:
         if rank == 0:
-            print(json.dumps(js_table(torch, fgd, dev, measured_peak())), flush=True)
+            print(json.dumps(js_table(torch, fgd, dev, measured_peak(), U=args.js_positions)), flush=True)
         return
     if args.sweep:
         if rank == 0:
@@ -654,9 +655,12 @@ def js_table(torch, fgd, dev, peak, K=8, U=4096, V=128256, k=100, reps=5):
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / reps
-    nbytes = U * V * 4 + (K + 1) * U * k * 32      # gathers move one 32-byte sector per entry
+    nbytes = U * V * 4 + (K + 1) * U * k * 32      # one read of the averaged logits + one 32-byte sector per gathered entry
+    gbs = nbytes / (ms * 1e-3) / 1e9
     return {"metric": "js_token_positions_per_s", "value": U / (ms * 1e-3), "ms": ms, "K": K, "U": U, "V": V, "top_k": k,
-            "algorithmic_gb": nbytes / 1e9, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak[0],
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak[0], "unit": "GB/s", "frac": gbs / peak[0],
+                         "algorithmic_bytes": nbytes, "peak_kind": f"of {peak[1]}", "traffic": None,
+                         "kernel": "js_select_stream_kernel (+ js_distance_kernel, js_mean_kernel: the whole call is timed)"},
             "cd_js": float(cdw.mean())}
 
 

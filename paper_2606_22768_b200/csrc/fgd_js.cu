@@ -4,13 +4,16 @@
 // (exact radix select, ties to the lower token index); every worker's distribution and the
 // averaged model's are restricted to those tokens, renormalised, and compared with the
 // normalised Jensen-Shannon distance sqrt(JS / ln 2), all in float64 in the log domain.
-// Two kernels: one CTA per position selects the tokens, one warp per (worker, position) pair
-// evaluates the distance; a third sums the distances of each worker in a fixed order.
+// Kernels: one CTA per position selects the tokens in a single pass over the row (rows that defeat
+// its sampling bound are redone by an exact multi-pass select), one warp per (worker, position)
+// pair evaluates the distance, and a last kernel sums the distances of each worker in a fixed order.
 #include <cuda_runtime.h>
 
 #include <cstdio>
 
 #include "fgd_internal.h"
+#include "fgd_nvtx.h"
+#include "fgd_step_dense_tc.cuh"   // mbarrier / shared-memory helpers
 
 using namespace fgd;
 
@@ -28,15 +31,271 @@ int js_fail(int status, const char* fmt, ...) {
 }
 
 // fp32 -> unsigned key whose ASCENDING order is DESCENDING float order (largest logit first).
+// (ascending key = negative ? ~b : b | sign; its complement in two operations)
 __device__ __forceinline__ uint32_t desc_key(float x) {
   const uint32_t b = __float_as_uint(x);
-  const uint32_t asc = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-  return ~asc;
+  const uint32_t neg = (uint32_t)((int32_t)b >> 31);      // all ones for a negative value
+  return b ^ (~neg & 0x7FFFFFFFu);
 }
 
-// One CTA per row: indices of the k smallest keys (= k largest logits), ascending index order.
+// ---------------------------------------------------------------------------------------------
+// Streaming select: ONE pass over the row in HBM.
+//
+// A lower bound of the k-th largest logit of the whole row comes from a sample: every thread takes
+// the largest of its 16 elements of the row's first kSample, and the k-th largest of those 1024
+// maxima bounds the row's k-th largest from below (k distinct elements reach it).  The bound is
+// taken on a 13-bit histogram of the ordered keys (sign, exponent, four mantissa bits), i.e. it is a
+// bin: every element whose bin lies beyond that boundary bin is out for certain.  The row is then
+// streamed once; the rare elements that pass (under one percent of a row in random order) are
+// appended to a candidate list in shared memory, and the exact answer -- the k smallest
+// (key, index) pairs, i.e. ties to the lower token index -- is found among the candidates: a second
+// histogram over them gives the row's true boundary bin, whatever lies before it is selected, and
+// each member of the boundary bin counts how many members precede it as a (key, index) pair to
+// learn whether it is among the few still needed; the k indices find their output slots the same
+// way (rank by counting: no sorting network, no barriers).
+// A row that defeats the sample (ascending order, huge groups of equal logits) overflows a list; it
+// is then marked (first output index -1) and redone by the exact multi-pass kernel below.
+// The row travels through a ring of shared-memory stages filled by 1-D bulk copies (TMA) that a
+// producer warp keeps in flight, so the bytes in flight do not depend on the consumers' registers;
+// the first stages double as the sample (they are looked at twice without being loaded twice).
+constexpr int kStrConsumers = 512;             // consumer threads; one more warp produces
+constexpr int kStrBlock = kStrConsumers + 32;
+constexpr int kBinShift = 20;                  // key >> 20: 4096 bins (sign, exponent, three mantissa bits)
+constexpr int kBins = 1 << (32 - kBinShift);
+constexpr int kChunk = 4096;                   // floats per stage (16 KB)
+constexpr int kStrStages = 4;                  // the ring; also the sample (16 K elements)
+constexpr int kCand = 2048;                    // candidate list entries
+constexpr int kBnd = 512;                      // boundary-bin list entries
+constexpr size_t kStrSmem = 128 + sizeof(float) * kChunk * kStrStages + sizeof(unsigned) * kBins +
+                            sizeof(unsigned long long) * (kCand + kBnd) + sizeof(int) * kMaxTopK;
+constexpr uint32_t kStrSpin = 1u << 22;        // polls before a wait gives up (the row is then redone by the exact kernel)
+
+__device__ __forceinline__ bool js_wait(uint32_t bar, uint32_t parity, const int* abort_flag) {
+  for (uint32_t it = 0; it < kStrSpin; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 31u) == 31u && *(const volatile int*)abort_flag) return false;
+  }
+  return false;
+}
+
+// One lane polls, the warp follows (far fewer polls competing with the other CTA's arithmetic).
+__device__ __forceinline__ bool js_warp_wait(uint32_t bar, uint32_t parity, const int* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = js_wait(bar, parity, abort_flag) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// First bin b with cum(b) >= k over hist[kBins]; the kStrConsumers consumer threads call (named
+// barrier 1).  *bin_out, *before_out: that bin and the count of the bins before it; untouched when
+// the histogram holds fewer than k entries.
+__device__ __forceinline__ void find_boundary_bin(const unsigned* hist, unsigned k, unsigned* warp_tot, unsigned* bin_out,
+                                                  unsigned* before_out, int tid) {
+  constexpr int PER = kBins / kStrConsumers;
+  const int lane = tid & 31, warp = tid >> 5;
+  unsigned loc[PER], sum = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) { loc[j] = hist[tid * PER + j]; sum += loc[j]; }
+  unsigned incl = sum;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  named_bar_sync(1, kStrConsumers);
+  unsigned before = incl - sum;
+  for (int w = 0; w < warp; ++w) before += warp_tot[w];
+  if (before < k && before + sum >= k) {       // exactly one thread, unless the total is below k
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if (before < k && before + loc[j] >= k) { *bin_out = (unsigned)(tid * PER + j); *before_out = before; }
+      before += loc[j];
+    }
+  }
+  named_bar_sync(1, kStrConsumers);
+}
+
+__global__ void __launch_bounds__(kStrBlock)
+js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t* __restrict__ idx_out) {
+  extern __shared__ __align__(128) unsigned char js_smem[];
+  __shared__ __align__(8) unsigned long long bars[2 * kStrStages];     // full[], empty[]
+  __shared__ unsigned warp_tot[kStrConsumers / 32];
+  __shared__ unsigned s_bin, s_before, s_ncand, s_nbnd, s_nfin;
+  __shared__ int abort_flag;
+  unsigned char* base = js_smem + ((128u - (smem_u32(js_smem) & 127u)) & 127u);
+  float* ring = reinterpret_cast<float*>(base);
+  unsigned* hist = reinterpret_cast<unsigned*>(ring + (size_t)kChunk * kStrStages);
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(hist + kBins);
+  unsigned long long* bnd = cand + kCand;
+  int* fin = reinterpret_cast<int*>(bnd + kBnd);
+  const float* row = avg_logits + (size_t)blockIdx.x * V;
+  int32_t* out = idx_out + (size_t)blockIdx.x * k;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[kStrStages]);
+
+  // the 16-byte aligned body of the row goes through the ring; up to three elements before and
+  // after it are read directly
+  int64_t head = (int64_t)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(row) & 15u)) & 15u) >> 2);
+  if (head > V) head = V;
+  const int64_t body = (V - head) / 4 * 4;                 // floats
+  const int64_t nchunks = (body + kChunk - 1) / kChunk;
+  const int nres = (int)(nchunks < kStrStages ? nchunks : kStrStages);   // chunks resident at the start = the sample
+
+  if (tid == 0) {
+    for (int s = 0; s < kStrStages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, kStrConsumers / 32);   // one arrival per consumer warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_bin = kBins - 1; s_before = 0; s_ncand = 0; s_nbnd = 0; s_nfin = 0;
+    abort_flag = 0;
+  }
+  for (int i = tid; i < kBins; i += kStrBlock) hist[i] = 0;
+  __syncthreads();
+
+  if (warp == kStrConsumers / 32) {
+    // ===================================================== producer (one elected lane)
+    if (lane == 0) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      int64_t c = 0;
+      bool ok = true;
+      for (; c < nchunks; ++c) {
+        const int s = (int)(c % kStrStages);
+        if (c >= kStrStages) ok = js_wait(bar_empty + 8u * s, (uint32_t)(c / kStrStages - 1) & 1, &abort_flag);
+        if (!ok) break;
+        const int64_t left = body - c * kChunk;
+        const uint32_t bytes = (uint32_t)((left < kChunk ? left : kChunk) * sizeof(float));
+        mbar_expect_tx(bar_full + 8u * s, bytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                     ::"r"(smem_u32(ring + (size_t)s * kChunk)), "l"(row + head + c * kChunk), "r"(bytes), "r"(bar_full + 8u * s), "l"(policy)
+                     : "memory");
+      }
+      if (!ok) *(volatile int*)&abort_flag = 1;
+      // never exit under a copy in flight: bounded wait for the last use of every stage
+      for (int64_t j = (c > kStrStages ? c - kStrStages : 0); j < c; ++j) {
+        const uint32_t bar = bar_full + 8u * (uint32_t)(j % kStrStages), parity = (uint32_t)(j / kStrStages) & 1;
+        for (uint32_t it = 0; it < kStrSpin; ++it) {
+          uint32_t done;
+          asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+          if (done) break;
+        }
+      }
+    }
+    return;
+  }
+
+  // ===================================================== consumers
+  bool failed = false;
+  // ---- sample: the largest element each thread sees in the resident chunks
+  uint32_t best = 0xFFFFFFFFu;                       // smallest key = largest logit
+  bool have = false;
+  for (int c = 0; c < nres && !failed; ++c) {
+    if (!js_warp_wait(bar_full + 8u * c, 0, &abort_flag, lane)) { failed = true; break; }
+    const int64_t left = body - (int64_t)c * kChunk;
+    const int n4 = (int)((left < kChunk ? left : kChunk) / 4);
+    const float4* src = reinterpret_cast<const float4*>(ring + (size_t)c * kChunk);
+    for (int j = tid; j < n4; j += kStrConsumers) {
+      const float4 t = src[j];
+      best = min(min(best, desc_key(t.x)), min(desc_key(t.y), min(desc_key(t.z), desc_key(t.w))));
+      have = true;
+    }
+  }
+  if (have) atomicAdd(&hist[best >> kBinShift], 1u);
+  if (failed) *(volatile int*)&abort_flag = 1;
+  named_bar_sync(1, kStrConsumers);
+  find_boundary_bin(hist, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
+  const unsigned b0 = s_bin;
+  const uint32_t key_max = b0 >= (unsigned)(kBins - 1) ? 0xFFFFFFFFu : (((b0 + 1u) << kBinShift) - 1u);   // largest key inside bin b0
+
+  // ---- the one pass over the row: keep what is not beyond the sample's boundary bin
+  auto consider = [&](float x, int64_t i) {
+    const uint32_t key = desc_key(x);
+    if (key <= key_max) {
+      const unsigned slot = atomicAdd(&s_ncand, 1u);
+      if (slot < (unsigned)kCand) cand[slot] = ((unsigned long long)key << 32) | (unsigned long long)(uint32_t)i;
+    }
+  };
+  if (tid < head) consider(row[tid], tid);
+  if (head + body + tid < V) consider(row[head + body + tid], head + body + tid);
+  for (int64_t c = 0; c < nchunks && !*(volatile int*)&abort_flag; ++c) {
+    const int s = (int)(c % kStrStages);
+    if (c >= nres && !js_warp_wait(bar_full + 8u * s, (uint32_t)(c / kStrStages) & 1, &abort_flag, lane)) {
+      *(volatile int*)&abort_flag = 1;
+      break;
+    }
+    const int64_t left = body - c * kChunk;
+    const int n4 = (int)((left < kChunk ? left : kChunk) / 4);
+    const float4* src = reinterpret_cast<const float4*>(ring + (size_t)s * kChunk);
+    const int64_t i0 = head + c * kChunk;
+#pragma unroll 2
+    for (int j = tid; j < n4; j += kStrConsumers) {
+      const float4 t = src[j];
+      consider(t.x, i0 + 4 * j);
+      consider(t.y, i0 + 4 * j + 1);
+      consider(t.z, i0 + 4 * j + 2);
+      consider(t.w, i0 + 4 * j + 3);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_empty + 8u * s);
+  }
+  for (int i = tid; i < kBins; i += kStrConsumers) hist[i] = 0;
+  named_bar_sync(1, kStrConsumers);
+  const unsigned ncand = s_ncand;
+  if (*(volatile int*)&abort_flag || ncand > (unsigned)kCand) {   // a wait gave up, or the sample's bound was too weak for this row
+    if (tid == 0) out[0] = -1;
+    return;
+  }
+  // ---- exact boundary bin of the whole row, from the candidates
+  for (unsigned i = tid; i < ncand; i += kStrConsumers) atomicAdd(&hist[(unsigned)(cand[i] >> (32 + kBinShift))], 1u);
+  named_bar_sync(1, kStrConsumers);
+  find_boundary_bin(hist, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
+  const unsigned b1 = s_bin, above = s_before, nb = hist[b1];
+  if (nb > (unsigned)kBnd) {                     // too many logits in one bin (large groups of equal values)
+    if (tid == 0) out[0] = -1;
+    return;
+  }
+  for (unsigned i = tid; i < ncand; i += kStrConsumers) {
+    const unsigned long long e = cand[i];
+    const unsigned bin = (unsigned)(e >> (32 + kBinShift));
+    if (bin < b1) fin[atomicAdd(&s_nfin, 1u)] = (int)(uint32_t)e;            // selected for certain (above < k of them)
+    else if (bin == b1) bnd[atomicAdd(&s_nbnd, 1u)] = e;
+  }
+  named_bar_sync(1, kStrConsumers);
+  // of the boundary bin's nb members the `need` smallest (key, index) pairs are taken: larger logit
+  // first, then the lower index.  All pairs are distinct, so a member's rank is the count of smaller ones.
+  const unsigned need = (unsigned)k - above;     // 1 <= need <= nb
+  for (unsigned i = tid; i < nb; i += kStrConsumers) {
+    const unsigned long long e = bnd[i];
+    unsigned rank = 0;
+    for (unsigned j = 0; j < nb; ++j) rank += bnd[j] < e ? 1u : 0u;
+    if (rank < need) fin[above + rank] = (int)(uint32_t)e;
+  }
+  named_bar_sync(1, kStrConsumers);
+  // ---- output in ascending index order: the slot of an index is the count of smaller selected indices
+  if (tid < k) {
+    const int mine = fin[tid];
+    int rank = 0;
+    for (int j = 0; j < k; ++j) rank += fin[j] < mine ? 1 : 0;
+    out[rank] = mine;
+  }
+}
+
+// Exact multi-pass select (four 8-bit radix passes and an ordered compaction), one CTA per row.
+// Rows the streaming kernel could not finish are marked with a first index of -1; with
+// `only_marked` every other row returns at once.
 __global__ void __launch_bounds__(kSelBlock)
-js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t* __restrict__ idx_out) {
+js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t* __restrict__ idx_out, int only_marked) {
+  if (only_marked && idx_out[(size_t)blockIdx.x * k] != -1) return;     // (uniform for the CTA)
   __shared__ unsigned int hist[256];
   __shared__ unsigned int s_prefix, s_remaining, s_less;
   __shared__ unsigned int warp_tot[2][kSelBlock / 32];
@@ -194,16 +453,26 @@ js_mean_kernel(const double* __restrict__ d_js, int64_t U, double* __restrict__ 
 extern "C" int fgd_js_distance(int device, int K, int64_t U, int64_t V, int top_k, const float* worker_logits,
                                const float* avg_logits, int32_t* top_idx, double* d_js, double* cd_worker,
                                void* stream) {
+  FGD_NVTX_RANGE("fgd_js_distance");
   if (K < 1 || K > FGD_MAX_K || U < 1 || V < 1 || top_k < 1 || top_k > kMaxTopK || top_k > V)
     return js_fail(FGD_ERR_INVALID_ARG, "fgd_js_distance: need 1 <= K <= %d, U, V >= 1, 1 <= top_k <= min(%d, V)", FGD_MAX_K, kMaxTopK);
-  if (U * (int64_t)K > 0x7fffffff * 8ll || U > 0x7fffffff)
+  if (U * (int64_t)K > 0x7fffffff * 8ll || U > 0x7fffffff || V > 0x7fffffff)
     return js_fail(FGD_ERR_INVALID_ARG, "fgd_js_distance: too many positions");
   if (!worker_logits || !avg_logits || !top_idx || !d_js || !cd_worker) return js_fail(FGD_ERR_INVALID_ARG, "fgd_js_distance: NULL pointer");
   int prev = -1;
   if (cudaGetDevice(&prev) != cudaSuccess) return js_fail(FGD_ERR_CUDA, "cudaGetDevice failed");
   if (prev != device && cudaSetDevice(device) != cudaSuccess) return js_fail(FGD_ERR_CUDA, "cannot select device %d", device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  js_select_kernel<<<(unsigned)U, kSelBlock, 0, st>>>(avg_logits, V, top_k, top_idx);
+  static bool smem_set[64] = {};
+  if (device < 64 && !smem_set[device]) {
+    if (cudaFuncSetAttribute(js_select_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStrSmem) != cudaSuccess) {
+      if (prev != device) cudaSetDevice(prev);
+      return js_fail(FGD_ERR_CUDA, "fgd_js_distance: cannot size the select kernel's shared memory");
+    }
+    smem_set[device] = true;
+  }
+  js_select_stream_kernel<<<(unsigned)U, kStrBlock, kStrSmem, st>>>(avg_logits, V, top_k, top_idx);
+  js_select_kernel<<<(unsigned)U, kSelBlock, 0, st>>>(avg_logits, V, top_k, top_idx, 1);   // rows the stream kernel marked
   const int64_t pairs = (int64_t)K * U;
   js_distance_kernel<<<(unsigned)((pairs + 7) / 8), 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
   js_mean_kernel<<<K, 32, 0, st>>>(d_js, U, cd_worker);

@@ -58,13 +58,32 @@ def test_top_tokens_and_truncated_metric():
 
 # ------------------------------------------------------------------ GPU parity
 @pytest.mark.gpu
-@pytest.mark.parametrize("K,U,V,k", [(4, 64, 32000, 100), (8, 33, 5001, 100), (2, 7, 100, 100), (3, 5, 70000, 37), (1, 1, 256, 1)])
-def test_js_distance_gpu(K, U, V, k):
+@pytest.mark.parametrize("K,U,V,k,shape", [
+    (4, 64, 32000, 100, "plain"), (8, 33, 5001, 100, "plain"), (2, 7, 100, 100, "plain"), (3, 5, 70000, 37, "plain"),
+    (1, 1, 256, 1, "plain"), (2, 9, 128256, 100, "plain"), (2, 6, 40003, 256, "plain"),
+    (8, 33, 5001, 100, "equal_below_cut"),   # many equal logits in the averaged model, below the cut
+    (2, 8, 5001, 100, "tie_at_cut"),         # 101 equal logits above everything else: the cut falls inside the group
+    (2, 6, 30000, 100, "big_tie_at_cut"),    # 4286 equal top logits: more than the streaming kernel's boundary list holds
+    (2, 5, 70000, 100, "ascending"),         # rows in ascending order: the sampling bound is useless, candidates overflow
+    (1, 3, 20000, 64, "all_equal"),
+    (2, 4, 50001, 100, "descending"),
+])
+def test_js_distance_gpu(K, U, V, k, shape):
     import torch
     import paper_2606_22768_b200 as fgd
     work, avg = _logits(K, U, V, seed=3)
-    if V == 5001:                      # force ties at the cut: many equal logits in the averaged model
+    if shape == "equal_below_cut":
         avg[:, ::7] = 1.25
+    elif shape == "tie_at_cut":
+        avg[:, ::50] = 11.0
+    elif shape == "big_tie_at_cut":
+        avg[:, ::7] = 11.0
+    elif shape == "ascending":
+        avg = np.sort(avg, axis=1)
+    elif shape == "descending":
+        avg = np.ascontiguousarray(np.sort(avg, axis=1)[:, ::-1])
+    elif shape == "all_equal":
+        avg[:] = 0.5
     w = torch.from_numpy(work).cuda()
     a = torch.from_numpy(avg).cuda()
     idx = torch.full((U, k), -1, dtype=torch.int32, device="cuda")
