@@ -189,7 +189,16 @@ int kt_of(int K) {
 }
 // The TMA-pipelined fused step is also instantiated for 3, 6 and 12 workers (clusters that are not
 // a power of two); the stand-alone kernels and the register path run those with run-time K.
-int kt_tma_of(int K) { return (K == 3 || K == 6 || K == 12) ? K : kt_of(K); }
+// The worker counts in between run zero-padded on the next of those kernels: 5 on 6, 7 on 8, 9-11 on
+// 12, 13-15 on 16 (the padded rows never touch HBM).
+int kt_tma_of(int K) {
+  if (K == 3 || K == 6 || K == 12) return K;
+  if (K == 5) return 6;
+  if (K == 7) return 8;
+  if (K >= 9 && K <= 11) return 12;
+  if (K >= 13 && K <= 15) return 16;
+  return kt_of(K);
+}
 int want_vec(int KT) { return KT == 0 ? 1 : (KT <= 16 ? 4 : (KT == 32 ? 2 : 1)); }
 
 // Calls f.template operator()<KT, VEC>() for the (KT, VEC) pair chosen at run time.

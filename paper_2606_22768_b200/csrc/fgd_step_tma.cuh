@@ -85,7 +85,12 @@ constexpr int kMaxStages = 8;
 // D2T: compile-time neighbour count of a gather Mix2 (-1 = read at run time; ignored for a mean
 // or dense Mix2).
 // D1T: the same for a fused gather Mix1 (-1 = run time).
-template <int KT, int VEC, int CONSUMERS, bool DENSE2, int D2T, int D1T, typename M2>
+// PAD: the worker count KR = a.K is smaller than the compile-time KT and the problem is zero-padded
+// to KT rows: the TMA boxes are KT rows tall (rows at or beyond KR lie outside the tensor and arrive
+// as zeros without touching HBM), the padded rows of every mix carry zero weights, and loads of a
+// matrix-valued x, all stores and the consensus terms are predicated on the row being real.  Worker
+// counts 5, 7, 9-11 and 13-15 run this way on the 6, 8, 12 and 16-worker kernels.
+template <int KT, int VEC, int CONSUMERS, bool DENSE2, int D2T, int D1T, typename M2, bool PAD = false>
 // (for 3, 6 and 12 workers the compiler is told that one CTA per SM is all there will be -- the
 // stage ring takes the shared memory -- which frees it from a self-imposed register target:
 // K = 12 5.5 -> 6.2 TB/s; for the other counts the same hint measured 0-1.5 % slower)
@@ -105,7 +110,9 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
   __shared__ double red[NWARP][FGD_MAX_K];
 
   const StepArgs& a = ta.s;
-  const int K = KT > 0 ? KT : a.K;
+  const int K = KT > 0 ? KT : a.K;                 // rows of a tile
+  const int KR = PAD ? a.K : K;                    // real workers (<= K)
+  static_assert(!PAD || KT > 0, "padding needs a compile-time worker count");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool want_cd = a.partials != nullptr;
   const int NT = ta.n_tensors;
@@ -130,14 +137,21 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if constexpr (DENSE2) {
-    for (int i = tid; i < K * K; i += CONSUMERS + 32) wts[i] = m2.Wt[i];
+    if constexpr (PAD) {                            // m2.Wt is packed with stride KR: zero rows / columns beyond it
+      for (int i = tid; i < K * K; i += CONSUMERS + 32) {
+        const int n = i / K, m = i % K;
+        wts[i] = (n < KR && m < KR) ? m2.Wt[n * KR + m] : 0.f;
+      }
+    } else {
+      for (int i = tid; i < K * K; i += CONSUMERS + 32) wts[i] = m2.Wt[i];
+    }
   }
   __syncthreads();
 
-  constexpr int KR = KT > 0 ? KT : 1;
-  float sacc[KR];
+  constexpr int KS = KT > 0 ? KT : 1;
+  float sacc[KS];
 #pragma unroll
-  for (int m = 0; m < KR; ++m) sacc[m] = 0.f;
+  for (int m = 0; m < KS; ++m) sacc[m] = 0.f;
 
   if (warp == CONSUMERS / 32) {
     // ===================================================== producer warp (one elected lane)
@@ -181,7 +195,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
     if constexpr (KT == 0) {
       for (int m = 0; m < K; ++m) sas[m * CONSUMERS + tid] = 0.f;
     }
-    const float invK = 1.0f / (float)K;
+    const float invK = 1.0f / (float)KR;
     const float lr = a.lr, mu = a.mu;
     // A matrix-valued Mix1 result is used only by the thread that owns the column, so with a
     // compile-time K it is not staged: each thread prefetches its K rows of the NEXT tile
@@ -194,10 +208,10 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
       const int64_t c_ = tile_ * T + (int64_t)tid * VEC;
       if (tile_ < ntiles && c_ + VEC <= P) {
 #pragma unroll
-        for (int m = 0; m < KX; ++m) dst[m] = ld_stream<VEC>(a.x + (size_t)m * ld + c_);
+        for (int m = 0; m < KX; ++m) dst[m] = (!PAD || m < KR) ? ld_stream<VEC>(a.x + (size_t)m * ld + c_) : p_zero<VEC>();
       } else if (tile_ < ntiles && c_ < P) {
         for (int m = 0; m < KX; ++m)
-          for (int q = 0; q < VEC; ++q) dst[m].v[q] = c_ + q < P ? a.x[(size_t)m * ld + c_ + q] : 0.f;
+          for (int q = 0; q < VEC; ++q) dst[m].v[q] = (c_ + q < P && (!PAD || m < KR)) ? a.x[(size_t)m * ld + c_ + q] : 0.f;
       }
     };
     if (x_direct) fetch_x(blockIdx.x, xr_next);
@@ -309,6 +323,10 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
           else v = a.avg_momentum ? vbar : SCol<VEC>::ld(C, m * TPB + t);
           const Pack<VEC> vn = p_fma<VEC>(v, mu, gh);                       // v' = mu v + ghat
           const Pack<VEC> tn = p_fma<VEC>(p_fma<VEC>(vn, mu, gh), -lr, xm);   // x - lr (ghat + mu v')
+          if (PAD && m >= KR) {                 // a padded row: nothing to store, nothing to count
+            if constexpr (REGS) av[m] = p_zero<VEC>();
+            return;
+          }
           asum = p_add<VEC>(asum, tn);
           if (whole) {
             st_stream<VEC>(mom_col + off, vn);
@@ -358,7 +376,7 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
               for (int q = 0; q < VEC; ++q)
                 if (col + q >= P) d.v[q] = 0.f;
             }
-            const float sq = p_hsum<VEC>(p_fma<VEC>(d, d, p_zero<VEC>()));
+            const float sq = p_hsum<VEC>(p_fma<VEC>(d, d, p_zero<VEC>()));      // (sums of padded rows are never read)
             if constexpr (KT > 0) sacc[m] += sq;
             else sas[m * CONSUMERS + tid] += sq;
           }
@@ -391,13 +409,13 @@ outer_step_tma_kernel(const TmaStepArgs ta, const M2 m2, const GatherMix m1,
     }
   }
   __syncthreads();
-  if (want_cd && tid < K) {
+  if (want_cd && tid < KR) {
     double d = 0.0;
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) d += red[w][tid];
-    a.partials[(size_t)blockIdx.x * K + tid] = d;
+    a.partials[(size_t)blockIdx.x * KR + tid] = d;
   }
-  if (want_cd) finalize_in_last_cta(a.partials, K, a.cd_out, a.done);
+  if (want_cd) finalize_in_last_cta(a.partials, KR, a.cd_out, a.done);
 }
 
 }  // namespace fgd

@@ -7,7 +7,8 @@ using namespace fgd;
 namespace {
 static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, const GatherMix& g2, const DenseMix& d2,
                     const GatherMix& g1, TmaShape sh, cudaStream_t st, int* grid_out) {
-  const int K = c->K, KT = kt_tma_of(K);
+  const int KT = kt_tma_of(c->K), K = KT > 0 ? KT : c->K;      // K: rows of a tile; KT > c->K: zero-padded worker count
+  const bool pad = KT > 0 && KT != c->K;
   TmaStepArgs ta;
   ta.s = a;
   ta.status = c->status;
@@ -18,10 +19,10 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
   const int T = sh.consumers * sh.vec;
   const int boxc = T < 256 ? T : 256;
   CUtensorMap tp, tl, tm, tx;
-  if (int rc = make_tensor_map(c, &tp, a.theta_prev, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tl, a.theta_local, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tm, a.momentum, boxc)) return rc;
-  if (int rc = make_tensor_map(c, &tx, a.xsrc == XSRC_MATRIX ? a.x : a.theta_prev, boxc)) return rc;
+  if (int rc = make_tensor_map(c, &tp, a.theta_prev, boxc, K)) return rc;
+  if (int rc = make_tensor_map(c, &tl, a.theta_local, boxc, K)) return rc;
+  if (int rc = make_tensor_map(c, &tm, a.momentum, boxc, K)) return rc;
+  if (int rc = make_tensor_map(c, &tx, a.xsrc == XSRC_MATRIX ? a.x : a.theta_prev, boxc, K)) return rc;
   const size_t smem = tma_fixed_smem(K, KT, dense2, sh.consumers) + tma_stage_bytes(K, T, ta.n_tensors) * sh.stages;
   const int64_t ntiles = (c->P + T - 1) / T;
   // neighbour count of a gather Mix2 as a template argument when it is one of the common ones
@@ -39,14 +40,31 @@ static int launch_step_tma_group(fgd_ctx* c, const StepArgs& a, bool dense2, con
                        (g1.D == d2t || (g1.D == 3 && d2t == 4) || (g1.D > 4 && d2t == 8));
   auto go = [&]<int KTc, int VECc, int Cc, int D2c, bool SAME1>() -> int {
     int grid = 0;
+    constexpr bool kPadBuilt = KTc == 6 || KTc == 8 || KTc == 12 || KTc == 16;   // kernels that also exist zero-padded
     if constexpr (D2c == -2) {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, true, -1, -1, DenseMix>;
-      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, Cc + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
+      auto launch = [&](auto kern) -> int {
+        if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
+        kern<<<grid, Cc + 32, smem, st>>>(ta, d2, g1, tp, tl, tm, tx);
+        return FGD_OK;
+      };
+      if constexpr (kPadBuilt) {
+        if (pad) { if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, true, -1, -1, DenseMix, true>)) return r; }
+        else if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, true, -1, -1, DenseMix>)) return r;
+      } else {
+        if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, true, -1, -1, DenseMix>)) return r;
+      }
     } else {
-      auto kern = outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, (SAME1 ? D2c : -1), GatherMix>;
-      if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
-      kern<<<grid, Cc + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
+      auto launch = [&](auto kern) -> int {
+        if (int r = persistent_grid(c, kern, Cc + 32, smem, ntiles, &grid)) return r;
+        kern<<<grid, Cc + 32, smem, st>>>(ta, g2, g1, tp, tl, tm, tx);
+        return FGD_OK;
+      };
+      if constexpr (kPadBuilt) {
+        if (pad) { if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, (SAME1 ? D2c : -1), GatherMix, true>)) return r; }
+        else if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, (SAME1 ? D2c : -1), GatherMix>)) return r;
+      } else {
+        if (int r = launch(outer_step_tma_kernel<KTc, VECc, Cc, false, D2c, (SAME1 ? D2c : -1), GatherMix>)) return r;
+      }
     }
     *grid_out = grid;
     return check_launch(c, "outer_step_tma_kernel");

@@ -71,7 +71,7 @@ bool tma_eligible(const fgd_ctx* c, const StepArgs& a, bool dense2, bool heavy, 
   if (c->ld % 4 != 0 || c->P >= (int64_t)0x7fffffff - 4096) return false;
   if (!aligned16(a.theta_prev) || !aligned16(a.theta_local) || !aligned16(a.momentum) || !aligned16(a.theta_new)) return false;
   if (a.xsrc == XSRC_MATRIX && !aligned16(a.x)) return false;
-  const int K = c->K, KT = kt_tma_of(K), NT = tma_n_tensors(a, KT, dense2);
+  const int KT = kt_tma_of(c->K), K = KT > 0 ? KT : c->K, NT = tma_n_tensors(a, KT, dense2);   // K: rows of a tile (padded)
   const size_t budget = (size_t)c->max_smem_optin - 6144;  // static shared memory (barriers, reduction buffer) + slack
   for (const auto& sh : kTmaShapes) {
     if (sh[0] != KT) continue;

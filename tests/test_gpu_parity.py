@@ -149,6 +149,18 @@ STEP_CASES = [
     (24, 7000, ("mean",), ("dense", gen.sinkhorn_W(5, 24))),
     (17, 6002, ("matching",), ("ring",)),
     (40, 3000, ("mean",), ("mean",)),
+    # worker counts zero-padded onto the 6, 8, 12 and 16-worker fp32 kernels (5; 7; 9-11; 13-15)
+    (5, 70001, ("mean",), ("ring",)),
+    (5, 9000, ("ring", 0.2), ("ring", 0.2)),
+    (7, 40002, ("mean",), ("dense", gen.sinkhorn_W(2, 7))),
+    (7, 30000, ("matching",), ("randgraph", 3, 0.2)),
+    (9, 30001, ("ring",), ("ring",)),
+    (10, 50003, ("mean",), ("randgraph", 5)),
+    (11, 20000, ("randgraph", 4, 0.1), ("circulant", 3)),
+    (13, 40001, ("mean",), ("dense", gen.sinkhorn_W(6, 13))),
+    (14, 30002, ("circulant", 2, 0.2), ("circulant", 2, 0.2)),
+    (15, 60000, ("mean",), ("circulant", 4)),
+    (15, 3, ("ring",), ("ring",)),
     # gossip Mix1 fused into the tensor-core kernel (gathered from the staged theta_prev)
     (64, 5001, ("hypercube", 0.1), ("hypercube", 0.1)),
     (64, 4000, ("ring",), ("dense", SINK64)),
@@ -343,6 +355,8 @@ VARIANTS = [
     ("ring40-GlobalM1S", 40, 4001, ("mean",), ("ring",), False, True),
     ("dense48-subset", 48, 6000, ("mean",), ("dense", gen.sinkhorn_W(3, 48)), True, False),
     ("ring24-subset-GlobalM1S", 24, 9000, ("mean",), ("ring",), True, True),
+    ("ring13-subset-GlobalM1S-padded", 13, 30000, ("mean",), ("ring",), True, True),
+    ("dense10-subset-padded", 10, 20000, ("mean",), ("dense", gen.sinkhorn_W(8, 10)), True, False),
 ]
 
 
@@ -453,6 +467,7 @@ def test_argument_errors():
     (8, 20000, ("mean",), ("matching", 0.05), 60),                          # the paper's setting, many rounds
     (64, 6000, ("ring", 0.1), ("dense", gen.sinkhorn_W(0, 64)), 30),        # tensor-core step and mix
     (48, 5000, ("mean",), ("ring",), 40),                                   # padded tensor-core shape
+    (13, 30000, ("ring", 0.1), ("ring", 0.1), 30),                          # zero-padded onto the 16-worker fp32 kernel
 ])
 def test_long_free_running_rounds(K, P, mix1, mix2, rounds):
     """Many free-running rounds (the oracle keeps its own float64 state): the fp32 path must not drift
