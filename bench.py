@@ -354,6 +354,29 @@ def time_rounds(torch, st, steps, warmup, min_seconds=0.0, graph=None, barrier=N
             "clocks": clocks}
 
 
+def pattern_probe(torch, fgd, st, reps=5):
+    """Time of the arithmetic-free tile copy that moves the fused step's bytes (3 [K,P] tensors read,
+    2 written, the step's own tile shape) on this configuration's tensors, in this run: the roofline
+    of the step's access pattern on this machine.  None for worker counts the probe is not built for."""
+    if st.K not in (4, 8, 16, 32, 64):
+        return None
+    f = lambda: fgd.fgd_debug_stream_pattern(st.drv.ctx, st.local, st.theta, st.mom, st.theta)
+    for _ in range(2):
+        f()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(st.main)
+        f()
+        b.record(st.main)
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = statistics.mean(ts)
+    return {"ms": ms, "ms_min": min(ts), "bytes": 20 * st.K * st.P, "gbs": 20 * st.K * st.P / (ms * 1e-3) / 1e9,
+            "what": "fgd_debug_stream_pattern: the step's tiles and TMA ring, no arithmetic, in place"}
+
+
 def roofline_of(cfg, cfg_id, K, P, kern_times, fuse_mix1, peak, peak_kind, traffic_ok=True):
     x_vec = cfg["mix1"][0] == "mean"
     step_bytes = (20 * K * P + 4 * P) if x_vec else 24 * K * P      # outer-step kernel, algorithmic
@@ -414,6 +437,10 @@ def extra_configs(torch, fgd, gen, inputs_gpu, OuterRound, dev, local_rank, peak
                  "frac_of_nominal_8000": roof["frac_of_nominal_8000"], "traffic": roof["traffic"],
                  "ms_per_round": ms_round, "rounds_timed": t["rounds"], "gpu_launches": t["launches"],
                  "worker_params_per_s": st.K * st.P / (ms_round * 1e-3)}
+        if cfg_id != 1:
+            entry["pattern"] = pattern_probe(torch, fgd, st)
+            if entry["pattern"]:
+                entry["frac_of_pattern"] = entry["pattern"]["gbs"] and entry["achieved"] / entry["pattern"]["gbs"]
         if cfg_id == 1:
             entry["note"] = "working set fits in L2: a latency configuration, achieved/frac are not HBM figures"
             entry["latency"] = latency_leg(torch, fgd, st.drv, cfg, st.theta, st.local, st.mom, st.seed, st.dense_W, dev)
@@ -522,6 +549,7 @@ def run_ours(args):
     if rank == 0:
         # context: the same STREAM-style copy the pool's peak was measured with, on THIS box, now
         roofline["copy_gbs_this_box"] = copy_bandwidth(torch, dev)
+        roofline["pattern"] = pattern_probe(torch, fgd, st)      # and the step's own access pattern without arithmetic
     if rank == 0 and 3 * K * P * 4 <= 4 * 126e6:
         line["latency"] = latency_leg(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, dev)
     if rank == 0 and not args.no_overlap:

@@ -112,6 +112,17 @@ int64_t fgd_launch_count(const fgd_ctx* ctx);
  * Both stay set until changed.  Not for production use. */
 typedef enum { FGD_DEBUG_SPIN_LIMIT = 1, FGD_DEBUG_SKIP_TILE = 2 } fgd_debug_key;
 int fgd_debug_set(fgd_ctx* ctx, int key, int64_t value);
+/* Measurement aid (no counterpart in the paper): the HBM traffic of fgd_outer_step without its
+ * arithmetic.  Reads theta_local, theta_prev and momentum and writes theta_new and momentum in the
+ * fused step's own tiles (all K rows by a few hundred columns, the same TMA stage ring), storing
+ * theta_prev's values into theta_new and the momentum's own values back: on an in-place call
+ * (theta_new == theta_prev) no tensor changes.  Its time on the caller's tensors is the roofline of
+ * the step's ACCESS PATTERN (3 K row streams read and 2 K written concurrently), which lies below
+ * a plain copy's bandwidth, the more so the larger K is.  Device [K, ld] tensors as in
+ * fgd_outer_step, same aliasing rules; needs the TMA path's alignment (else FGD_ERR_UNSUPPORTED);
+ * built for K = 4, 8, 16, 32, 64. */
+int fgd_debug_stream_pattern(fgd_ctx* ctx, const float* theta_local, const float* theta_prev, float* momentum,
+                             float* theta_new, void* stream);
 
 /* ---- mixing operators (Sec. 3 "Gossip-based Mixing"; App. A table of (Mix1, Mix2)) ---- */
 typedef enum {

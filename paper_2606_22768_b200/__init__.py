@@ -66,6 +66,7 @@ def _load():
         "fgd_set_path": (i32, [vp, i32]),
         "fgd_device_status": (i32, [vp, vp]),
         "fgd_debug_set": (i32, [vp, i32, i64]),
+        "fgd_debug_stream_pattern": (i32, [vp, vp, vp, vp, vp, vp]),
         "fgd_outer_grad": (i32, [vp, vp, vp, vp, vp]),
         "fgd_mix": (i32, [vp, descp, vp, vp, i32, vp]),
         "fgd_outer_step": (i32, [vp, descp, descp, vp, i32, vp, vp, vp, vp, dbl, dbl, vp, vp]),
@@ -283,6 +284,14 @@ FGD_DEBUG_SPIN_LIMIT, FGD_DEBUG_SKIP_TILE = 1, 2
 def fgd_debug_set(ctx: Context, key: int, value: int) -> None:
     """Test hooks of the bounded device-side waits (see ``include/fgd.h``)."""
     ctx._check(_lib.fgd_debug_set(ctx._h, int(key), int(value)))
+
+
+def fgd_debug_stream_pattern(ctx: Context, theta_local, theta_prev, momentum, theta_new, stream=None) -> None:
+    """The fused step's HBM traffic without its arithmetic (a measurement aid, see ``include/fgd.h``)."""
+    ctx._check(_lib.fgd_debug_stream_pattern(ctx._h, _dev_ptr(theta_local, "theta_local", "torch.float32"),
+                                             _dev_ptr(theta_prev, "theta_prev", "torch.float32"),
+                                             _dev_ptr(momentum, "momentum", "torch.float32"),
+                                             _dev_ptr(theta_new, "theta_new", "torch.float32"), _stream(stream)))
 
 
 def fgd_device_status(ctx: Context, stream=None) -> None:
