@@ -4,6 +4,7 @@
 
 #include "fgd_mix_dense_tc.cuh"
 #include "fgd_step_dense_tc.cuh"
+#include "fgd_step_gossip_tc.cuh"
 #include "fgd_tma_host.h"
 
 using namespace fgd;
@@ -53,10 +54,23 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
   switch (xm) {
     case 1: return full ? launch(outer_step_dense_tc_kernel<KP, 1, true>) : launch(outer_step_dense_tc_kernel<KP, 1, false>);
     case 2:
-      if constexpr (KP == 32)    // two consumer groups where the registers allow it
+      // A sparse Mix1 fused.  At the 64-worker shape both mixes run as MMAs with the operands in tensor
+      // memory (fgd_step_gossip_tc.cuh: ring + ring fused 4.3 -> 4.6 TB/s at K = 64); at the 32- and
+      // 48-worker shapes the per-tile latencies of that chain weigh more than the gathers it saves
+      // (K = 32: 4.0 against 5.2 TB/s, K = 48: 4.2 against 4.3), so those keep the gather from the stage.
+      if constexpr (KP == 64) {
+        auto launch_g = [&](auto kern) -> int {
+          const int block = TcGossipShape<KP>::kThreads;
+          if (int r = persistent_grid(c, kern, block, TcGossipShape<KP>::kSmem, ntiles, grid)) return r;
+          kern<<<*grid, block, TcGossipShape<KP>::kSmem, st>>>(ta, d2, g1, tp, tl, tm);
+          return FGD_OK;
+        };
+        return full ? launch_g(outer_step_gossip_tc_kernel<KP, true>) : launch_g(outer_step_gossip_tc_kernel<KP, false>);
+      } else if constexpr (KP == 32) {   // two consumer groups where the registers allow it
         return full ? launch(outer_step_dense_tc_kernel<KP, 2, true, false, 2>, 2) : launch(outer_step_dense_tc_kernel<KP, 2, false, false, 2>, 2);
-      else
+      } else {
         return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
+      }
     default:
       if (a.n_ranges != 0)
         return full ? launch(outer_step_dense_tc_kernel<KP, 0, true, true>) : launch(outer_step_dense_tc_kernel<KP, 0, false, true>);

@@ -67,6 +67,35 @@ def test_fused_step_wait_runs_out_and_context_recovers(K, P, mix2):
     assert not torch.equal(th, th0)                        # and it did compute something
 
 
+def test_gossip_tensor_core_step_wait_runs_out_and_context_recovers():
+    """The step with a sparse Mix1 fused (both mixes as MMAs, ring of single boxes)."""
+    K, P = 64, 148 * 4 * 128 + 36
+    m1, m2 = fgd.MixDesc.ring(K), fgd.MixDesc.hypercube(K)
+    th0, loc0, mom0 = _inputs(K, P, 33)
+
+    def run(ctx, th, mom):
+        cd = torch.zeros(K, dtype=torch.float64, device="cuda")
+        fgd.fgd_outer_step(ctx, m2, m1, None, False, loc0, th, mom, th, 0.7, 0.9, cd)
+        return cd
+
+    ctx = fgd.Context(K, P)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SPIN_LIMIT, SPIN)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SKIP_TILE, 1)
+    run(ctx, th0.clone(), mom0.clone())
+    _expect_timeout_once(ctx)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SPIN_LIMIT, 0)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SKIP_TILE, -1)
+    th, mom = th0.clone(), mom0.clone()
+    cd = run(ctx, th, mom)
+    fgd.fgd_device_status(ctx)
+    fresh = fgd.Context(K, P)
+    th_f, mom_f = th0.clone(), mom0.clone()
+    cd_f = run(fresh, th_f, mom_f)
+    fgd.fgd_device_status(fresh)
+    assert torch.equal(th, th_f) and torch.equal(mom, mom_f) and torch.equal(cd, cd_f)
+    assert not torch.equal(th, th0)
+
+
 def test_tensor_core_mix_wait_runs_out_and_context_recovers():
     K, P = 64, 148 * 4 * 128 + 36
     W = fgd.MixDesc.dense(gen.sinkhorn_W(5, K))
