@@ -283,13 +283,22 @@ outer_step_dense_tc_kernel(const TmaStepArgs ta, const DenseMix m2, const Gather
     // instruction descriptor: D fp32, A and B tf32, both K-major, N = K, M = 128
     constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(K >> 3) << 17) | ((uint32_t)(T >> 4) << 24);
     int64_t i = gid;                               // the CTA's i-th tile; group g takes i = g, g + NG, ...
-    for (int64_t tile = blockIdx.x + (int64_t)gid * gridDim.x; tile < ntiles; tile += (int64_t)NG * gridDim.x, i += NG) {
+    // A one-value-per-column x is requested a whole tile ahead: under a saturated memory system a plain
+    // load waits in the same queues as the TMA boxes for several microseconds, longer than the part of a
+    // tile that precedes its first use.
+    const int64_t tile_step = (int64_t)NG * gridDim.x;
+    float x_ahead = 0.f;
+    {
+      const int64_t col0 = (blockIdx.x + (int64_t)gid * gridDim.x) * T + c;
+      if (a.xsrc == XSRC_VECTOR && col0 < P) x_ahead = __ldcs(a.x + col0);
+    }
+    for (int64_t tile = blockIdx.x + (int64_t)gid * gridDim.x; tile < ntiles; tile += tile_step, i += NG) {
       const int s = (int)(i % STAGES);
       const uint32_t use = (uint32_t)(i / STAGES);
       const int64_t col = tile * T + c;
       const bool live = col < P;
-      float xv = 0.f;
-      if (a.xsrc == XSRC_VECTOR && live) xv = __ldcs(a.x + col);
+      float xv = x_ahead;
+      if (a.xsrc == XSRC_VECTOR && col + tile_step * T < P) x_ahead = __ldcs(a.x + col + tile_step * T);
       float xr[XM == 1 ? H : 1];                   // a matrix-valued Mix1 result: this thread's rows, requested
       if constexpr (XM == 1) {                     // now so that they arrive behind the TMA wait and the MMA
         if (live) {
