@@ -389,6 +389,8 @@ __device__ __forceinline__ double warp_sum(double v) {   // fixed butterfly: eve
 }
 
 // One warp per (worker m, position u): normalised JS distance over the selected tokens.
+// PER = tokens per lane (k <= 32 PER): the register arrays are sized for the k in use.
+template <int PER>
 __global__ void __launch_bounds__(256)
 js_distance_kernel(const float* __restrict__ worker_logits, const float* __restrict__ avg_logits,
                    const int32_t* __restrict__ idx, int K, int64_t U, int64_t V, int k, double* __restrict__ d_js) {
@@ -399,7 +401,6 @@ js_distance_kernel(const float* __restrict__ worker_logits, const float* __restr
   const float* wrow = worker_logits + ((size_t)m * U + u) * V;
   const float* arow = avg_logits + (size_t)u * V;
   const int32_t* id = idx + (size_t)u * k;
-  constexpr int PER = kMaxTopK / 32;
   double p[PER], q[PER];
   double pmax = -1e300, qmax = -1e300;
 #pragma unroll
@@ -416,13 +417,19 @@ js_distance_kernel(const float* __restrict__ worker_logits, const float* __restr
   pmax = warp_max(pmax);
   qmax = warp_max(qmax);
   double ps = 0.0, qs = 0.0;
+  double ep[PER], eq[PER];                 // exp(logit - max): the probabilities up to their normalising sums
 #pragma unroll
   for (int j = 0; j < PER; ++j)
     if (lane + 32 * j < k) {
-      ps += exp(p[j] - pmax);
-      qs += exp(q[j] - qmax);
+      ep[j] = exp(p[j] - pmax);
+      eq[j] = exp(q[j] - qmax);
+      ps += ep[j];
+      qs += eq[j];
     }
-  const double plse = pmax + log(warp_sum(ps)), qlse = qmax + log(warp_sum(qs));
+  ps = warp_sum(ps);
+  qs = warp_sum(qs);
+  const double plse = pmax + log(ps), qlse = qmax + log(qs);
+  const double half_ip = 0.5 / ps, half_iq = 0.5 / qs;
   const double ln_half = -0.69314718055994530942;
   double js = 0.0;
 #pragma unroll
@@ -431,7 +438,7 @@ js_distance_kernel(const float* __restrict__ worker_logits, const float* __restr
       const double lp = p[j] - plse, lq = q[j] - qlse;
       const double hi = fmax(lp, lq), lo = fmin(lp, lq);
       const double lm = hi + log1p(exp(lo - hi)) + ln_half;      // log((p + q) / 2)
-      js += 0.5 * exp(lp) * (lp - lm) + 0.5 * exp(lq) * (lq - lm);
+      js += ep[j] * half_ip * (lp - lm) + eq[j] * half_iq * (lq - lm);   // 1/2 p (log p - log m) + 1/2 q (log q - log m)
     }
   js = warp_sum(js);
   if (lane == 0) d_js[pair] = sqrt(fmax(js, 0.0) / 0.69314718055994530942);
@@ -474,7 +481,11 @@ extern "C" int fgd_js_distance(int device, int K, int64_t U, int64_t V, int top_
   js_select_stream_kernel<<<(unsigned)U, kStrBlock, kStrSmem, st>>>(avg_logits, V, top_k, top_idx);
   js_select_kernel<<<(unsigned)U, kSelBlock, 0, st>>>(avg_logits, V, top_k, top_idx, 1);   // rows the stream kernel marked
   const int64_t pairs = (int64_t)K * U;
-  js_distance_kernel<<<(unsigned)((pairs + 7) / 8), 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
+  const unsigned grid_d = (unsigned)((pairs + 7) / 8);
+  if (top_k <= 32) js_distance_kernel<1><<<grid_d, 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
+  else if (top_k <= 64) js_distance_kernel<2><<<grid_d, 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
+  else if (top_k <= 128) js_distance_kernel<4><<<grid_d, 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
+  else js_distance_kernel<kMaxTopK / 32><<<grid_d, 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
   js_mean_kernel<<<K, 32, 0, st>>>(d_js, U, cd_worker);
   cudaError_t e = cudaGetLastError();
   if (prev != device) cudaSetDevice(prev);
