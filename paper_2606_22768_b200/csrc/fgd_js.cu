@@ -42,31 +42,40 @@ __device__ __forceinline__ uint32_t desc_key(float x) {
 // Streaming select: ONE pass over the row in HBM.
 //
 // A lower bound of the k-th largest logit of the whole row comes from a sample: every thread takes
-// the largest of its 16 elements of the row's first kSample, and the k-th largest of those 1024
-// maxima bounds the row's k-th largest from below (k distinct elements reach it).  The bound is
-// taken on a 13-bit histogram of the ordered keys (sign, exponent, four mantissa bits), i.e. it is a
-// bin: every element whose bin lies beyond that boundary bin is out for certain.  The row is then
-// streamed once; the rare elements that pass (under one percent of a row in random order) are
-// appended to a candidate list in shared memory, and the exact answer -- the k smallest
-// (key, index) pairs, i.e. ties to the lower token index -- is found among the candidates: a second
-// histogram over them gives the row's true boundary bin, whatever lies before it is selected, and
-// each member of the boundary bin counts how many members precede it as a (key, index) pair to
-// learn whether it is among the few still needed; the k indices find their output slots the same
-// way (rank by counting: no sorting network, no barriers).
+// the largest of its 24 elements of the row's first 12 K, and the k-th largest of those 512 maxima
+// bounds the row's k-th largest from below (k distinct elements reach it).  It is located on a 12-bit
+// histogram of the ordered keys (sign, exponent, three mantissa bits) and then sharpened to the exact
+// key by ranking the few maxima of the boundary bin.  The row is then streamed once; four elements at a
+// time are compared with the bound as floats, and the rare elements that reach it (about one percent
+// of a row in random order) are appended to a candidate list in shared memory.  The exact answer --
+// the k smallest (key, index) pairs, i.e. ties to the lower token index -- is found among the
+// candidates: a second histogram over them gives the row's true boundary bin, whatever lies before
+// it is selected, and each member of the boundary bin counts how many members precede it as a
+// (key, index) pair to learn whether it is among the few still needed; the k indices find their
+// output slots the same way (rank by counting: no sorting network).
 // A row that defeats the sample (ascending order, huge groups of equal logits) overflows a list; it
 // is then marked (first output index -1) and redone by the exact multi-pass kernel below.
-// The row travels through a ring of shared-memory stages filled by 1-D bulk copies (TMA) that a
+// The row travels through two 24 KB shared-memory stages filled by 1-D bulk copies (TMA) that a
 // producer warp keeps in flight, so the bytes in flight do not depend on the consumers' registers;
-// the first stages double as the sample (they are looked at twice without being loaded twice).
+// the first two stages double as the sample (they are looked at twice without being loaded twice).
+// Measured: the hand-off per stage, not the bytes, is what costs -- six 8 KB stages 0.84 ms, three
+// 16 KB 0.68 ms, two 24 KB 0.62 ms, one 48 KB 0.68 ms for the whole call at U = 4096 -- and three CTAs
+// per SM (69 KB each) beat two with a larger ring, because one row's start-up and candidate phases
+// then overlap two other rows' streaming.
 constexpr int kStrConsumers = 512;             // consumer threads; one more warp produces
 constexpr int kStrBlock = kStrConsumers + 32;
 constexpr int kBinShift = 20;                  // key >> 20: 4096 bins (sign, exponent, three mantissa bits)
 constexpr int kBins = 1 << (32 - kBinShift);
-constexpr int kChunk = 4096;                   // floats per stage (16 KB)
-constexpr int kStrStages = 4;                  // the ring; also the sample (16 K elements)
+constexpr int kChunk = 6144;                   // floats per stage (24 KB)
+constexpr int kStrStages = 2;                  // the ring; also the sample (12 K elements)
 constexpr int kCand = 2048;                    // candidate list entries
 constexpr int kBnd = 512;                      // boundary-bin list entries
-constexpr size_t kStrSmem = 128 + sizeof(float) * kChunk * kStrStages + sizeof(unsigned) * kBins +
+// The histogram has no memory of its own: for the sample it lies over the (still empty) candidate
+// list, for the candidates over the (by then idle) ring -- 69 KB per CTA, three CTAs per SM, so that one
+// row's start-up and candidate phases overlap two other rows' streaming.
+static_assert(sizeof(unsigned) * kBins <= sizeof(unsigned long long) * kCand && sizeof(unsigned) * kBins <= sizeof(float) * kChunk * kStrStages,
+              "the histogram must fit over the candidate list and over the ring");
+constexpr size_t kStrSmem = 128 + sizeof(float) * kChunk * kStrStages +
                             sizeof(unsigned long long) * (kCand + kBnd) + sizeof(int) * kMaxTopK;
 constexpr uint32_t kStrSpin = 1u << 22;        // polls before a wait gives up (the row is then redone by the exact kernel)
 
@@ -128,12 +137,13 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
   extern __shared__ __align__(128) unsigned char js_smem[];
   __shared__ __align__(8) unsigned long long bars[2 * kStrStages];     // full[], empty[]
   __shared__ unsigned warp_tot[kStrConsumers / 32];
-  __shared__ unsigned s_bin, s_before, s_ncand, s_nbnd, s_nfin;
+  __shared__ unsigned s_bin, s_before, s_ncand, s_nbnd, s_nfin, s_keymax;
   __shared__ int abort_flag;
   unsigned char* base = js_smem + ((128u - (smem_u32(js_smem) & 127u)) & 127u);
   float* ring = reinterpret_cast<float*>(base);
-  unsigned* hist = reinterpret_cast<unsigned*>(ring + (size_t)kChunk * kStrStages);
-  unsigned long long* cand = reinterpret_cast<unsigned long long*>(hist + kBins);
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(ring + (size_t)kChunk * kStrStages);
+  unsigned* const hist_sample = reinterpret_cast<unsigned*>(cand);     // before any candidate exists
+  unsigned* const hist_cand = reinterpret_cast<unsigned*>(ring);       // after the last chunk has been read
   unsigned long long* bnd = cand + kCand;
   int* fin = reinterpret_cast<int*>(bnd + kBnd);
   const float* row = avg_logits + (size_t)blockIdx.x * V;
@@ -158,7 +168,7 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
     s_bin = kBins - 1; s_before = 0; s_ncand = 0; s_nbnd = 0; s_nfin = 0;
     abort_flag = 0;
   }
-  for (int i = tid; i < kBins; i += kStrBlock) hist[i] = 0;
+  for (int i = tid; i < kBins; i += kStrBlock) hist_sample[i] = 0;
   __syncthreads();
 
   if (warp == kStrConsumers / 32) {
@@ -209,13 +219,44 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
       have = true;
     }
   }
-  if (have) atomicAdd(&hist[best >> kBinShift], 1u);
+  if (have) atomicAdd(&hist_sample[best >> kBinShift], 1u);
   if (failed) *(volatile int*)&abort_flag = 1;
   named_bar_sync(1, kStrConsumers);
-  find_boundary_bin(hist, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
+  find_boundary_bin(hist_sample, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
   const unsigned b0 = s_bin;
-  const uint32_t key_max = b0 >= (unsigned)(kBins - 1) ? 0xFFFFFFFFu : (((b0 + 1u) << kBinShift) - 1u);   // largest key inside bin b0
+  // The bound is sharpened from "bin b0" to the exact key inside it: the maxima that fall into b0 (a
+  // handful) are listed and the (k - before)-th smallest of them, found by counting ranks, is the
+  // k-th largest maximum itself.  (If the list overflows the whole bin stays in.)
+  const unsigned need0 = (unsigned)k - s_before, nb0 = hist_sample[b0];
+  uint32_t* const lst = reinterpret_cast<uint32_t*>(bnd);
+  if (tid == 0) s_keymax = b0 >= (unsigned)(kBins - 1) ? 0xFFFFFFFFu : (((b0 + 1u) << kBinShift) - 1u);   // largest key inside bin b0
+  named_bar_sync(1, kStrConsumers);
+  const bool refine = b0 < (unsigned)(kBins - 1) && nb0 >= need0 && nb0 <= (unsigned)(2 * kBnd);
+  const bool mine_in = refine && have && (best >> kBinShift) == b0;
+  if (mine_in) lst[atomicAdd(&s_nbnd, 1u)] = best;
+  named_bar_sync(1, kStrConsumers);
+  if (mine_in) {
+    unsigned smaller = 0, equal = 0;
+    for (unsigned j = 0; j < nb0; ++j) {
+      const uint32_t o = lst[j];
+      smaller += o < best ? 1u : 0u;
+      equal += o == best ? 1u : 0u;
+    }
+    if (smaller < need0 && smaller + equal >= need0) s_keymax = best;     // every thread that hits it writes the same key
+  }
+  named_bar_sync(1, kStrConsumers);
+  const uint32_t key_max = s_keymax;
+  if (tid == 0) s_nbnd = 0;
 
+  // The same bound as a float: the smallest value of bin b0.  Four elements at a time are tested against
+  // it with one comparison of their maximum; only the rare group that reaches it is looked at element
+  // by element with the exact key test.  (NaN logits are not supported: fmaxf drops them.)
+  float thr;
+  {
+    const uint32_t bits = (key_max & 0x80000000u) ? key_max : (key_max ^ 0x7FFFFFFFu);   // inverse of desc_key
+    thr = __uint_as_float(bits);
+    if (key_max == 0xFFFFFFFFu || thr != thr) thr = key_max == 0xFFFFFFFFu ? -__int_as_float(0x7f800000) : __int_as_float(0x7f800000);
+  }
   // ---- the one pass over the row: keep what is not beyond the sample's boundary bin
   auto consider = [&](float x, int64_t i) {
     const uint32_t key = desc_key(x);
@@ -239,16 +280,18 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
 #pragma unroll 2
     for (int j = tid; j < n4; j += kStrConsumers) {
       const float4 t = src[j];
-      consider(t.x, i0 + 4 * j);
-      consider(t.y, i0 + 4 * j + 1);
-      consider(t.z, i0 + 4 * j + 2);
-      consider(t.w, i0 + 4 * j + 3);
+      if (fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)) >= thr) {
+        consider(t.x, i0 + 4 * j);
+        consider(t.y, i0 + 4 * j + 1);
+        consider(t.z, i0 + 4 * j + 2);
+        consider(t.w, i0 + 4 * j + 3);
+      }
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar_empty + 8u * s);
+    __syncwarp();                                   // (reads through the generic proxy are ordered before the
+    if (lane == 0) mbar_arrive(bar_empty + 8u * s); //  refill by the arrive / wait pair itself: no proxy fence)
   }
-  for (int i = tid; i < kBins; i += kStrConsumers) hist[i] = 0;
+  named_bar_sync(1, kStrConsumers);               // every consumer is through with the ring
+  for (int i = tid; i < kBins; i += kStrConsumers) hist_cand[i] = 0;
   named_bar_sync(1, kStrConsumers);
   const unsigned ncand = s_ncand;
   if (*(volatile int*)&abort_flag || ncand > (unsigned)kCand) {   // a wait gave up, or the sample's bound was too weak for this row
@@ -256,10 +299,10 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
     return;
   }
   // ---- exact boundary bin of the whole row, from the candidates
-  for (unsigned i = tid; i < ncand; i += kStrConsumers) atomicAdd(&hist[(unsigned)(cand[i] >> (32 + kBinShift))], 1u);
+  for (unsigned i = tid; i < ncand; i += kStrConsumers) atomicAdd(&hist_cand[(unsigned)(cand[i] >> (32 + kBinShift))], 1u);
   named_bar_sync(1, kStrConsumers);
-  find_boundary_bin(hist, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
-  const unsigned b1 = s_bin, above = s_before, nb = hist[b1];
+  find_boundary_bin(hist_cand, (unsigned)k, warp_tot, &s_bin, &s_before, tid);
+  const unsigned b1 = s_bin, above = s_before, nb = hist_cand[b1];
   if (nb > (unsigned)kBnd) {                     // too many logits in one bin (large groups of equal values)
     if (tid == 0) out[0] = -1;
     return;
@@ -292,16 +335,12 @@ js_select_stream_kernel(const float* __restrict__ avg_logits, int64_t V, int k, 
 
 // Exact multi-pass select (four 8-bit radix passes and an ordered compaction), one CTA per row.
 // Rows the streaming kernel could not finish are marked with a first index of -1; with
-// `only_marked` every other row returns at once.
-__global__ void __launch_bounds__(kSelBlock)
-js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t* __restrict__ idx_out, int only_marked) {
-  if (only_marked && idx_out[(size_t)blockIdx.x * k] != -1) return;     // (uniform for the CTA)
+// `only_marked` every other row is skipped.
+__device__ __forceinline__ void js_select_row(const float* __restrict__ row, int64_t V, int k, int32_t* __restrict__ out) {
   __shared__ unsigned int hist[256];
   __shared__ unsigned int s_prefix, s_remaining, s_less;
   __shared__ unsigned int warp_tot[2][kSelBlock / 32];
   __shared__ unsigned int s_eq_base, s_sel_base;
-  const float* row = avg_logits + (size_t)blockIdx.x * V;
-  int32_t* out = idx_out + (size_t)blockIdx.x * k;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     s_prefix = 0;
@@ -374,6 +413,16 @@ js_select_kernel(const float* __restrict__ avg_logits, int64_t V, int k, int32_t
       s_sel_base += sel_total;
     }
     __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(kSelBlock)
+js_select_kernel(const float* __restrict__ avg_logits, int64_t U, int64_t V, int k, int32_t* __restrict__ idx_out, int only_marked) {
+  // a small grid walks the rows: with `only_marked` almost every row costs one load of its marker
+  for (int64_t u = blockIdx.x; u < U; u += gridDim.x) {
+    if (only_marked && idx_out[(size_t)u * k] != -1) continue;          // (uniform for the CTA)
+    js_select_row(avg_logits + (size_t)u * V, V, k, idx_out + (size_t)u * k);
+    __syncthreads();                                                    // the shared state is free for the next row
   }
 }
 
@@ -479,7 +528,7 @@ extern "C" int fgd_js_distance(int device, int K, int64_t U, int64_t V, int top_
     smem_set[device] = true;
   }
   js_select_stream_kernel<<<(unsigned)U, kStrBlock, kStrSmem, st>>>(avg_logits, V, top_k, top_idx);
-  js_select_kernel<<<(unsigned)U, kSelBlock, 0, st>>>(avg_logits, V, top_k, top_idx, 1);   // rows the stream kernel marked
+  js_select_kernel<<<(unsigned)(U < 296 ? U : 296), kSelBlock, 0, st>>>(avg_logits, U, V, top_k, top_idx, 1);   // rows the stream kernel marked
   const int64_t pairs = (int64_t)K * U;
   const unsigned grid_d = (unsigned)((pairs + 7) / 8);
   if (top_k <= 32) js_distance_kernel<1><<<grid_d, 256, 0, st>>>(worker_logits, avg_logits, top_idx, K, U, V, top_k, d_js);
