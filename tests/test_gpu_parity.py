@@ -371,7 +371,8 @@ def test_paper_variants(name, K, P, mix1, mix2, subset, avg, path, mode):
 
 @pytest.mark.parametrize("K,P,mix2", [(16, 50001, ("ring",)), (8, 30000, ("xor",)), (64, 9000, ("dense", SINK64)),
                                        (64, 5000, ("hypercube",)), (6, 7000, ("ring",)), (2, 4000, ("ring",)),
-                                       (48, 6001, ("ring",)), (20, 5000, ("dense", gen.sinkhorn_W(6, 20)))])
+                                       (48, 6001, ("ring",)), (20, 5000, ("dense", gen.sinkhorn_W(6, 20))),
+                                       (13, 30001, ("ring",)), (10, 20000, ("randgraph", 3))])   # zero-padded fp32 shapes
 @pytest.mark.parametrize("path", PATHS)
 def test_step_emits_next_rounds_global_average(K, P, mix2, path):
     """Mix1 = global average chained through the fused step: round r writes x_{r+1} = mean(theta_new),
