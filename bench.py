@@ -88,6 +88,7 @@ def parse_args():
                     help="repeat the block of --steps rounds until the timed region lasts at least this long (0: exactly --steps rounds)")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table the default run appends")
     ap.add_argument("--js-positions", type=int, default=4096, help="with --js: token positions U (reduce for profiling)")
+    ap.add_argument("--jsonl", default="", help="write one JSON record per round of the untimed consensus trajectory to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true")
@@ -396,22 +397,45 @@ def roofline_of(cfg, cfg_id, K, P, kern_times, fuse_mix1, peak, peak_kind, traff
     return roof, step_bytes, mix1_bytes
 
 
-def consensus_trajectory(torch, fgd, inputs_gpu, st, rounds):
+def consensus_trajectory(torch, fgd, inputs_gpu, st, rounds, jsonl_path=None):
     """The configuration's own rounds from its initial state with a fresh drift every round (untimed):
-    the consensus distance (Sec. 4.4 definition) after each.  Restores nothing: call it last."""
+    the consensus distance (Sec. 4.4 definition) after each.  Restores nothing: call it last.
+    With `jsonl_path` one record per round goes to that file: the per-worker sums of squares, both
+    consensus distances, the fused step's time and bandwidth, and how many edges each mix lost."""
     inputs_gpu.theta0(st.theta, st.seed)
     st.mom.zero_()
     st.drv._pending = None
-    out = []
+    out, records = [], []
+    K, P = st.K, st.P
+    x_vec = st.cfg["mix1"][0] == "mean"
+    step_bytes = 20 * K * P if st.flags.fuse_mix1 else ((20 * K * P + 4 * P) if x_vec else 24 * K * P)
+
+    def dropped(m):          # undirected edges the round's mask took out of a sparse mix
+        return 0 if m.edge_mask is None else int(((m.edge_mask == 0) & (m.nbr >= 0)).sum()) // 2
+
     for r in range(rounds):
+        m1, m2 = st.mix("mix1", r), st.mix("mix2", r)
         if not st.flags.fuse_mix1:
-            st.drv.launch_mix1(st.mix("mix1", r), st.theta)
+            st.drv.launch_mix1(m1, st.theta)
+            st.main.wait_event(st.drv._pending[0])
         inputs_gpu.local_steps(st.local, st.theta, st.sig, st.seed, r)
         st.drv.cd_sumsq = st.cd_log[r % st.cd_log.shape[0]]
-        st.drv.step(st.mix("mix2", r), st.local, st.theta, st.mom, st.theta, 0.7, 0.9,
-                    mix1_fused=st.mix("mix1", r) if st.flags.fuse_mix1 else None)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st.main)
+        st.drv.step(m2, st.local, st.theta, st.mom, st.theta, 0.7, 0.9, mix1_fused=m1 if st.flags.fuse_mix1 else None)
+        e1.record(st.main)
         torch.cuda.synchronize()
-        out.append(fgd.fgd_cd_finalize(st.drv.cd_sumsq.cpu().numpy())[0])
+        s = st.drv.cd_sumsq.cpu().numpy()
+        cd_norm, cd_sq = fgd.fgd_cd_finalize(s)
+        out.append(cd_norm)
+        ms = e0.elapsed_time(e1)
+        records.append({"round": r, "sumsq": [float(v) for v in s], "cd_norm": cd_norm, "cd_sq": cd_sq, "step_ms": ms,
+                        "step_gbs": step_bytes / (ms * 1e-3) / 1e9, "worker_params_per_s_step": K * P / (ms * 1e-3),
+                        "mix1_edges_dropped": dropped(m1), "mix2_edges_dropped": dropped(m2)})
+    if jsonl_path:
+        with open(jsonl_path, "w") as f:
+            for rec in records:
+                f.write(json.dumps(rec) + "\n")
     return out
 
 
@@ -561,7 +585,7 @@ def run_ours(args):
         line["e2e"] = e2e_leg(torch, dist, fgd, drv, cfg, theta, local, mom, st.cd_log, seed, dense_W, world, dev)
     if rank == 0 and graph is None and not args.chain_mix1:
         n = CONFIG_ROUNDS[args.config]
-        line["consensus"] = {"cd_norm_per_round": consensus_trajectory(torch, fgd, inputs_gpu, st, n), "rounds": n,
+        line["consensus"] = {"cd_norm_per_round": consensus_trajectory(torch, fgd, inputs_gpu, st, n, args.jsonl or None), "rounds": n,
                              "note": "separate untimed run of the configuration's own rounds from its initial state, fresh "
                                      "drift every round (the timed rounds reuse one theta_local: bandwidth only)"}
     del drv, theta, local, mom
