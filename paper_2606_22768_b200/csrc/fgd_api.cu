@@ -187,6 +187,26 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
     if (ok) return fgd_launch_mix_dense_tc(c, in, out, dm, st);
   }
 
+  // worker counts up to 16 that are not powers of two: compile-time kernels of their own (sparse and
+  // mean mixes, four columns per thread; run-time K before: ring 3.7-4.3 TB/s, mean 4.3-5.9)
+  if (!dense && small_odd_k(K) && pick_vec(4, c->P, c->ld, {in, out}) == 4) {
+    return dispatch_small_k(K, [&]<int KTc>() -> int {
+      const int64_t ntiles = (c->P + (int64_t)kBlock * 4 - 1) / ((int64_t)kBlock * 4);
+      const size_t smem = desc->kind == FGD_MIX_MEAN ? 0 : sizeof(float) * (size_t)K * kBlock * 4;
+      int grid = 0;
+      auto launch = [&](auto kern) -> int {
+        if (int rc = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return rc;
+        kern<<<grid, kBlock, smem, st>>>(a, gm);
+        return check_launch(c, "mix_kernel");
+      };
+      const int dt = (gm.kind == KMIX_GATHER && gm.D >= 1 && gm.D <= 4) ? (gm.D == 3 ? 4 : gm.D) : -1;
+      if (dt == 1) return launch(mix_kernel<KTc, 4, false, kBlock, GatherMix, 1>);
+      if (dt == 2) return launch(mix_kernel<KTc, 4, false, kBlock, GatherMix, 2>);
+      if (dt == 4) return launch(mix_kernel<KTc, 4, false, kBlock, GatherMix, 4>);
+      return launch(mix_kernel<KTc, 4, false, kBlock, GatherMix>);
+    });
+  }
+
   return dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);
     // the averaging path keeps everything in registers: no private columns, more CTAs per SM
@@ -414,6 +434,15 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
                         : launch(consensus_split_kernel<32, 2, 4, kSplitBlock>, ntiles))
       return r;
     return FGD_OK;
+  }
+  if (small_odd_k(K) && pick_vec(4, c->P, c->ld, {theta}) == 4) {   // compile-time kernels for 3, 5-7, 9-15 workers
+    return dispatch_small_k(K, [&]<int KTc>() -> int {
+      const int64_t ntiles = (c->P + (int64_t)kBlock * 4 - 1) / ((int64_t)kBlock * 4);
+      auto kern = consensus_kernel<KTc, 4, kBlock>;
+      if (int r = persistent_grid(c, kern, kBlock, 0, ntiles, &grid)) return r;
+      kern<<<grid, kBlock, 0, st>>>(theta, c->partials, K, c->P, c->ld, cd_sumsq, c->done);
+      return check_launch(c, "consensus_kernel");
+    });
   }
   int rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {
     const int64_t ntiles = (c->P + (int64_t)kBlock * VECc - 1) / ((int64_t)kBlock * VECc);

@@ -217,6 +217,19 @@ int dispatch_kv(int KT, int VEC, F&& f) {
   return FGD_ERR_UNSUPPORTED;
 }
 
+// The stand-alone mix and consensus kernels are also instantiated for the worker counts up to 16
+// that are not powers of two (four columns per thread only): calls f.template operator()<KT>().
+inline bool small_odd_k(int K) { return K >= 3 && K <= 15 && kt_of(K) == 0; }
+template <typename F>
+int dispatch_small_k(int K, F&& f) {
+#define FGD_CASE(kt) \
+  if (K == kt) return f.template operator()<kt>();
+  FGD_CASE(3) FGD_CASE(5) FGD_CASE(6) FGD_CASE(7) FGD_CASE(9) FGD_CASE(10) FGD_CASE(11)
+  FGD_CASE(12) FGD_CASE(13) FGD_CASE(14) FGD_CASE(15)
+#undef FGD_CASE
+  return FGD_ERR_UNSUPPORTED;
+}
+
 }  // namespace
 
 #endif

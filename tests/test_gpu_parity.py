@@ -58,6 +58,10 @@ MIX_CASES = [
     (48, 9001, ("ring",)), (40, 5000, ("dense", gen.sinkhorn_W(8, 40))), (33, 4100, ("matching",)), (63, 3000, ("mean",)),
     (32, 6002, ("dense", gen.sinkhorn_W(7, 32))), (24, 7000, ("ring", 0.3)), (17, 2000, ("dense", gen.sinkhorn_W(9, 17))),
     (64, 20000, ("hypercube", 0.1)), (8, 30000, ("hypercube", 0.2)), (16, 9000, ("randgraph", 5, 0.2)), (40, 3000, ("randgraph", 3)), (7, 2000, ("randgraph", 2)),
+    # every worker count up to 16 that is not a power of two has stand-alone kernels of its own
+    (3, 5001, ("ring",)), (6, 4100, ("matching",)), (6, 70001, ("ring", 0.2)), (7, 9000, ("ring",)), (10, 6000, ("randgraph", 3)),
+    (11, 3001, ("ring", 0.3, fgd.FGD_RENORM_SELF_ABSORB)), (12, 8000, ("matching",)), (13, 5000, ("randgraph", 5)),
+    (14, 4000, ("ring",)), (15, 7001, ("mean",)), (10, 2000, ("mean",)), (12, 3000, ("randgraph", 1)),
 ]
 
 
@@ -79,7 +83,8 @@ def test_mix_matrix_output(K, P, spec):
     assert torch.equal(f_in[:, :P], out)
 
 
-@pytest.mark.parametrize("K,P", [(4, 1 << 20), (16, 30001), (6, 513), (64, 4096), (64, 100004), (32, 65540), (32, 999)])
+@pytest.mark.parametrize("K,P", [(4, 1 << 20), (16, 30001), (6, 513), (64, 4096), (64, 100004), (32, 65540), (32, 999),
+                                 (6, 5120), (13, 40004), (11, 1000)])
 def test_mix_mean_vector_output(K, P):
     x = gen.theta0(4, K, P, 0.02, 5e-3)
     f_in, _ = upload(x, P)
@@ -94,7 +99,9 @@ def test_mix_mean_vector_output(K, P):
 # ------------------------------------------------------------------ fgd_consensus_distance
 @pytest.mark.parametrize("K,P,ld", [(4, 1 << 20, None), (16, 100001, 100004), (64, 20000, 20000), (32, 30002, 30002),
                                      (5, 7777, 7780), (1, 50, 50), (2, 3, 4), (64, 150004, 150016), (32, 200000, 200000),
-                                     (64, 131, 132), (32, 4, 4)])
+                                     (64, 131, 132), (32, 4, 4)]
+                         + [(K, 20000 + 37 * K, 20000 + 37 * K + (4 - (37 * K) % 4) % 4) for K in (3, 6, 7, 9, 10, 11, 12, 13, 14, 15)]
+                         + [(13, 5001, 5001)])      # odd row stride: the run-time-K kernel
 def test_consensus_distance(K, P, ld):
     ld = P if ld is None else ld
     th = gen.theta0(5, K, P, 0.02, 7e-4)
