@@ -650,7 +650,7 @@ def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
                 Ks=(2, 3, 4, 6, 8, 12, 16, 17, 24, 32, 40, 48, 56, 63, 64)):
     """Fused outer step (in place, consensus sums on) across worker counts at a fixed tensor size:
     Mix2 = ring / hypercube (powers of two) / dense Sinkhorn with x one value per column, and the
-    fully fused ring-ring round.  GB/s = algorithmic bytes (20 K P + 4 P, or 20 K P fused) / time."""
+    fully fused ring-ring and matching-matching (pairwise gossip for both mixes, App. A) rounds.  GB/s = algorithmic bytes (20 K P + 4 P, or 20 K P fused) / time."""
     out = {"peak_gbs": peak[0], "peak_kind": peak[1], "tensor_bytes": tensor_bytes, "unit": "GB/s", "rows": {}}
     for K in Ks:
         P = tensor_bytes // 4 // K // 128 * 128
@@ -661,7 +661,8 @@ def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
         cd = torch.zeros(K, dtype=torch.float64, device=dev)
         ctx = fgd.Context(K, P, device=dev.index or 0)
         ring = fgd.MixDesc.ring(K)
-        cases = {"ring": (ring, None), "dense": (fgd.MixDesc.dense(gen.sinkhorn_W(0, K)), None), "ring+ring fused": (ring, ring)}
+        cases = {"ring": (ring, None), "dense": (fgd.MixDesc.dense(gen.sinkhorn_W(0, K)), None), "ring+ring fused": (ring, ring),
+                 "matching+matching fused": (fgd.MixDesc.random_matching(K, 0, 0, 2), fgd.MixDesc.random_matching(K, 0, 0, 1))}
         if K & (K - 1) == 0 and K > 1:
             cases["hypercube"] = (fgd.MixDesc.hypercube(K), None)
         row = {}

@@ -278,11 +278,11 @@ def fgd_set_path(ctx: Context, path: int) -> None:
     ctx._check(_lib.fgd_set_path(ctx._h, int(path)))
 
 
-FGD_DEBUG_SPIN_LIMIT, FGD_DEBUG_SKIP_TILE = 1, 2
+FGD_DEBUG_SPIN_LIMIT, FGD_DEBUG_SKIP_TILE, FGD_DEBUG_GOSSIP_PATH = 1, 2, 3
 
 
 def fgd_debug_set(ctx: Context, key: int, value: int) -> None:
-    """Test hooks of the bounded device-side waits (see ``include/fgd.h``)."""
+    """Test and measurement hooks: bounded device-side waits, fused-gossip kernel choice (see ``include/fgd.h``)."""
     ctx._check(_lib.fgd_debug_set(ctx._h, int(key), int(value)))
 
 

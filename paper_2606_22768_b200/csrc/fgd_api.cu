@@ -110,6 +110,10 @@ int fgd_debug_set(fgd_ctx* c, int key, int64_t value) {
       if (value < -1 || value > 0x7fffffff) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: tile index %lld out of range", (long long)value);
       c->dbg_skip_tile = (int)value;
       return FGD_OK;
+    case FGD_DEBUG_GOSSIP_PATH:
+      if (value < 0 || value > 2) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: gossip path %lld out of range", (long long)value);
+      c->dbg_gossip_path = (int)value;
+      return FGD_OK;
     default:
       return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: unknown key %d", key);
   }
@@ -252,6 +256,36 @@ int fgd_outer_step(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix
                            cd_sumsq, nullptr, stream);
 }
 
+// Worker counts up to 15 that are not powers of two have a register kernel compiled for that very count
+// and a pipelined kernel that is either their own (3, 6, 12) or the next larger one run zero-padded (5 on 6,
+// 7 on 8, 9-11 on 12, 13-15 on 16), which moves no extra HBM bytes but does the larger kernel's
+// shared-memory traffic and arithmetic.  Which is faster was measured per structure (4 GB per tensor, in
+// place, consensus sums on; TB/s register / pipelined):
+//   9-11 workers: the register kernel everywhere (ring 5.96-6.00 / 4.7-5.5, dense 5.9 / 4.6-5.1, matrix x
+//   5.7-6.2 / 5.0-5.5, ring + ring fused 6.1-6.4 / 4.6-5.3, matching fused 6.3-6.4 / 4.6-5.5);
+//   6 and 12: their own pipelined kernel (6.0-6.6 / 5.4-6.3 the other way round);
+//   dense Mix2: register at 3, 7, 13-15 (5.9-6.2 / 4.2-5.9), a tie at 5;
+//   sparse Mix1 gathered in the kernel: register at 7 (6.0-6.4 / 4.8-5.7), at 5 from three neighbour slots
+//   (6.3 / 5.5; ring 5.8 / 6.2), at 14 and 15 up to two slots (5.4-6.0 / 4.9-5.6; four slots 4.7-4.9 / 4.9-5.9),
+//   pipelined at 3 and 13;
+//   matrix-valued x: register up to 7 workers (6.2-6.5 / 5.7-6.5), pipelined at 13-15 (4.7-5.9 / 5.3-5.7);
+//   x one value per column: register (5.9-6.3 / 5.2-5.9) except a light Mix2 at 7 (6.0 / 6.1-6.3).
+static bool reg_beats_pipelined(int K, bool dense2, bool x_matrix, bool gossip1, int D2, int D1) {
+  if (K == 6 || K == 12) return false;
+  if (K >= 9 && K <= 11) return true;
+  if (dense2) return K != 5;
+  const int D = D1 > D2 ? D1 : D2;
+  if (gossip1) {
+    if (K == 7) return true;
+    if (K == 5) return D >= 3;
+    if (K >= 14) return D <= 2;
+    return false;
+  }
+  if (x_matrix) return K <= 7;
+  if (K == 7) return D2 >= 3;
+  return true;
+}
+
 int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* mix1_fused, const float* x,
                       int x_is_vector, const float* theta_local, const float* theta_prev, float* momentum,
                       float* theta_new, double lr, double mu, double* cd_sumsq, const fgd_step_options* opts,
@@ -378,13 +412,34 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma))
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
+  const bool reg_odd = small_odd_k(K) && pick_vec(4, c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next}) == 4;
+  const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
+  const bool reg_odd_auto = reg_odd && reg_beats_pipelined(K, dense2, a.xsrc == XSRC_MATRIX, gossip1,
+                                                           dense2 ? 0 : g2.D, gossip1 ? g1.D : 0);
   if (can_tc && c->path != FGD_PATH_REGISTER) {
     rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
-  } else if (can_tma && c->path != FGD_PATH_REGISTER && !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && (KT == 8 || KT == 16))))) {
+  } else if (can_tma && c->path != FGD_PATH_REGISTER &&
+             !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && (KT == 8 || KT == 16)) || reg_odd_auto))) {
     // (AUTO keeps the register kernel with one or two workers, where a tile is too little work per
     // pipeline hand-off, and for a dense Mix2 at K = 8 and 16, where its all-register W g product
     // measured 5.9 / 6.1 TB/s against 5.2 / 5.0 TB/s for the shared-memory version of the pipelined kernel)
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
+  } else if (reg_odd) {
+    rc = dispatch_small_k(K, [&]<int KTc>() -> int {
+      const int64_t ntiles = (c->P + (int64_t)kBlock * 4 - 1) / ((int64_t)kBlock * 4);
+      const size_t col = sizeof(float) * (size_t)K * kBlock * 4;
+      const size_t smem = col + (a.stage_tp ? col : 0) + (dense2 ? sizeof(float) * (size_t)K * K : 0);
+      if (dense2) {
+        auto kern = outer_step_kernel<KTc, 4, true, kBlock, DenseMix>;
+        if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
+        kern<<<grid, kBlock, smem, st>>>(a, d2, g1);
+      } else {
+        auto kern = outer_step_kernel<KTc, 4, false, kBlock, GatherMix>;
+        if (int r = persistent_grid(c, kern, kBlock, smem, ntiles, &grid)) return r;
+        kern<<<grid, kBlock, smem, st>>>(a, g2, g1);
+      }
+      return check_launch(c, "outer_step_kernel");
+    });
   } else {
     const int vec = pick_vec(want_vec(KT), c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next});
     rc = dispatch_kv(KT, vec, [&]<int KTc, int VECc>() -> int {

@@ -36,6 +36,7 @@ struct fgd_ctx {
   int64_t launches = 0;
   uint32_t dbg_spin_limit = 0;   // fgd_debug_set: polls before a device-side wait gives up (0 = the default)
   int dbg_skip_tile = -1;        // fgd_debug_set: tile whose loads the pipelined kernels withhold (-1 = none)
+  int dbg_gossip_path = 0;       // fgd_debug_set: 0 = by slot count, 1 = gather, 2 = MMAs (tensor-core step, sparse Mix1 fused)
   char err[256] = "";
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
   // fgd_outer_step_from_host only (created by its first call): copy stream, one event per column
@@ -138,7 +139,9 @@ int ctas_per_sm(fgd_ctx* c, Kern kern, int block, size_t smem, int* out) {
     *out = it->second;
     return FGD_OK;
   }
-  if (smem > 48 * 1024)
+  cudaFuncAttributes fa;
+  FGD_CUDA(c, cudaFuncGetAttributes(&fa, kern));
+  if (smem + fa.sharedSizeBytes > 48 * 1024)     // the 48 KB default covers static + dynamic shared memory
     FGD_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int n = 0;
   FGD_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, block, smem));

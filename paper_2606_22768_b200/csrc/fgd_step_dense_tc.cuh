@@ -121,7 +121,7 @@ template <int DJ, int H, int T>
 // The H results go to this thread's tensor-memory scratch columns [tx, tx + H), eight at a time:
 // they are needed again only in the epilogue, and with all shared memory given to the stages a
 // spilled register goes all the way to L2.
-__device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A, int r0, int c, uint32_t tx) {
+__device__ __forceinline__ void tc_gather_x_rows(const GatherMix& m1, const float* A, int r0, int c, uint32_t tx) {
 #pragma unroll
   for (int mb = 0; mb < H; mb += 8) {
     float x8[8];
@@ -139,6 +139,15 @@ __device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A,
     tmem_st_8(tx + (uint32_t)mb, x8);
   }
   tmem_st_wait();
+}
+
+// The first row of the thread's half as a constant: every neighbour index and weight of the unrolled
+// gather is then read at a compile-time offset of the kernel's parameters (an immediate constant-bank
+// operand) instead of through an indexed constant load per slot and row.
+template <int DJ, int H, int T>
+__device__ __forceinline__ void tc_gather_x(const GatherMix& m1, const float* A, int r0, int c, uint32_t tx) {
+  if (r0 == 0) tc_gather_x_rows<DJ, H, T>(m1, A, 0, c, tx);
+  else tc_gather_x_rows<DJ, H, T>(m1, A, H, c, tx);
 }
 
 // XM: where the Mix1 result x comes from.  0 = one value per column (a given row, or the column

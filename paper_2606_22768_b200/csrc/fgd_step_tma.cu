@@ -54,11 +54,17 @@ static int launch_tc(fgd_ctx* c, const TmaStepArgs& ta, const DenseMix& d2, cons
   switch (xm) {
     case 1: return full ? launch(outer_step_dense_tc_kernel<KP, 1, true>) : launch(outer_step_dense_tc_kernel<KP, 1, false>);
     case 2:
-      // A sparse Mix1 fused.  At the 64-worker shape both mixes run as MMAs with the operands in tensor
-      // memory (fgd_step_gossip_tc.cuh: ring + ring fused 4.3 -> 4.6 TB/s at K = 64); at the 32- and
-      // 48-worker shapes the per-tile latencies of that chain weigh more than the gathers it saves
-      // (K = 32: 4.0 against 5.2 TB/s, K = 48: 4.2 against 4.3), so those keep the gather from the stage.
+      // A sparse Mix1 fused.  The gather from the stage costs one shared-memory load and one FMA per
+      // neighbour slot and row (indices and weights are immediate constant-bank operands); running Mix1
+      // as a second MMA group with the operands in tensor memory (fgd_step_gossip_tc.cuh) costs the
+      // same whatever the slot count.  Measured at K = 64, same mix on both sides, TB/s gather / MMAs:
+      // matching 5.24 / 4.69, ring 5.32 / 5.06, four slots 4.55 / 4.68, six (hypercube) 3.72 / 4.70 --
+      // so three slots and more take the MMAs.  At the 32- and 48-worker shapes the per-tile latencies
+      // of the MMA chain weigh more (K = 32: 4.0 TB/s against 4.7 for the gather at five slots).
       if constexpr (KP == 64) {
+        // one or two neighbour slots: the gather is cheaper than the second MMA group
+        if (c->dbg_gossip_path == 1 || (c->dbg_gossip_path == 0 && g1.D <= 2))
+          return full ? launch(outer_step_dense_tc_kernel<KP, 2, true>) : launch(outer_step_dense_tc_kernel<KP, 2, false>);
         auto launch_g = [&](auto kern) -> int {
           const int block = TcGossipShape<KP>::kThreads;
           if (int r = persistent_grid(c, kern, block, TcGossipShape<KP>::kSmem, ntiles, grid)) return r;

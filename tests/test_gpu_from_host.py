@@ -19,7 +19,8 @@ pytestmark = pytest.mark.gpu
     (16, 40000, ("hypercube", 0.1), ("hypercube", 0.1), 3, True),   # gossip Mix1 gathered in the kernel
     (64, 9000, ("mean",), ("dense", gen.sinkhorn_W(0, 64)), 4, False),   # tensor-core kernel per chunk
     (10, 50003, ("mean",), ("ring", 0.1), 5, False),             # zero-padded onto the 12-worker kernel
-    (64, 8000, ("ring",), ("hypercube",), 3, True),              # both mixes as MMAs per chunk
+    (64, 8000, ("hypercube",), ("ring",), 3, True),              # both mixes as MMAs per chunk
+    (64, 6000, ("matching",), ("hypercube",), 2, True),          # one neighbour slot: gathered from the stage
     (4, 3000, ("ring",), ("ring",), 1, False),                   # one chunk, matrix-valued x
 ])
 def test_outer_step_from_host(K, P, mix1, mix2, chunks, fused):

@@ -70,7 +70,7 @@ def test_fused_step_wait_runs_out_and_context_recovers(K, P, mix2):
 def test_gossip_tensor_core_step_wait_runs_out_and_context_recovers():
     """The step with a sparse Mix1 fused (both mixes as MMAs, ring of single boxes)."""
     K, P = 64, 148 * 4 * 128 + 36
-    m1, m2 = fgd.MixDesc.ring(K), fgd.MixDesc.hypercube(K)
+    m1, m2 = fgd.MixDesc.hypercube(K), fgd.MixDesc.ring(K)   # six neighbour slots: Mix1 runs as MMAs
     th0, loc0, mom0 = _inputs(K, P, 33)
 
     def run(ctx, th, mom):
