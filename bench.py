@@ -647,7 +647,7 @@ def kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, peak, r
 
 
 def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
-                Ks=(2, 3, 4, 6, 8, 12, 16, 17, 24, 32, 40, 48, 56, 63, 64)):
+                Ks=(2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 20, 24, 28, 32, 40, 48, 56, 63, 64)):
     """Fused outer step (in place, consensus sums on) across worker counts at a fixed tensor size:
     Mix2 = ring / hypercube (powers of two) / dense Sinkhorn with x one value per column, and the
     fully fused ring-ring and matching-matching (pairwise gossip for both mixes, App. A) rounds.  GB/s = algorithmic bytes (20 K P + 4 P, or 20 K P fused) / time."""

@@ -177,9 +177,17 @@ int fgd_mix(fgd_ctx* c, const fgd_mix_desc* desc, const float* in, float* out, i
     return K == 64 ? launch(mix_mean_split_kernel<64, 4, 4, kSplitBlock>) : launch(mix_mean_split_kernel<32, 2, 4, kSplitBlock>);
   }
 
+  // a sparse mix above 16 workers: the TMA-pipelined row gather, whatever the worker and slot counts
+  // (5.4-5.9 TB/s; the tensor-core mix on the densified matrix: 2.2-5.6, the 32- / 64-worker column kernels: 5.3 / 4.1)
+  if (!dense && !out_is_vector && gm.kind == KMIX_GATHER && K > 16 && c->path != FGD_PATH_REGISTER &&
+      fgd_mix_gather_tma_eligible(c, in, out))
+    return fgd_launch_mix_gather_tma(c, in, out, gm, st);
+
   // worker counts above 16 without a compile-time fp32 kernel, and dense matrices from K = 32 up:
   // the tensor-core kernel (any mix is a dense matrix, so a sparse or mean one is densified for it)
-  if (!out_is_vector && (c->path == FGD_PATH_AUTO || c->path == FGD_PATH_TMA) && fgd_mix_tc_eligible(c, in, dense)) {
+  // (not the global average: its load-and-add column kernel runs at 5.6-6.0 TB/s with any K, the densified one at 2.2-4.5)
+  if (!out_is_vector && desc->kind != FGD_MIX_MEAN && (c->path == FGD_PATH_AUTO || c->path == FGD_PATH_TMA) &&
+      fgd_mix_tc_eligible(c, in, dense)) {
     bool ok = true;
     if (!dense) {
       double Wd[FGD_MAX_K * FGD_MAX_K];
@@ -413,17 +421,27 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   const bool reg_odd = small_odd_k(K) && pick_vec(4, c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next}) == 4;
+  const bool reg_k = fgd_reg_k_built(K) && pick_vec(2, c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next}) == 2;
   const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
+  // 17-31 workers: the register kernel compiled for that count against the tensor-core kernel zero-padded to
+  // 32 (measured, TB/s register / tensor cores, K = 17 | 20 | 24 | 28): ring 6.0/5.2 | 6.0/5.9 | 5.6/5.7 | 5.7/5.6;
+  // four slots 5.9/4.9 | 5.8/4.9 | 4.8/5.8 | 5.0/5.5; matrix x 4.3/3.1 | 4.3/3.6 | 3.5/4.3 | 3.4/5.0; ring + ring fused
+  // 5.5/3.8 | 5.2/4.4 | 4.7/5.2 | 4.5/6.0; matching fused 6.2/3.8 | 5.7/4.3 | 5.4/5.1 | 5.0/5.9; dense 3.4/4.8 | 3.5/5.1.
+  const int gslots = (gossip1 && !dense2) ? (g1.D > g2.D ? g1.D : g2.D) : 0;
+  const bool reg_k_auto = reg_k && !dense2 && c->path == FGD_PATH_AUTO &&
+                          (K <= 20 || (gossip1 && ((gslots <= 1 && K <= 25) || (gslots <= 2 && K <= 21))));
   const bool reg_odd_auto = reg_odd && reg_beats_pipelined(K, dense2, a.xsrc == XSRC_MATRIX, gossip1,
                                                            dense2 ? 0 : g2.D, gossip1 ? g1.D : 0);
-  if (can_tc && c->path != FGD_PATH_REGISTER) {
+  if (can_tc && c->path != FGD_PATH_REGISTER && !reg_k_auto) {
     rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
-  } else if (can_tma && c->path != FGD_PATH_REGISTER &&
+  } else if (can_tma && c->path != FGD_PATH_REGISTER && !reg_k_auto &&
              !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && (KT == 8 || KT == 16)) || reg_odd_auto))) {
     // (AUTO keeps the register kernel with one or two workers, where a tile is too little work per
     // pipeline hand-off, and for a dense Mix2 at K = 8 and 16, where its all-register W g product
     // measured 5.9 / 6.1 TB/s against 5.2 / 5.0 TB/s for the shared-memory version of the pipelined kernel)
     rc = fgd_launch_step_tma(c, a, dense2, g2, d2, g1, shape, st, &grid);
+  } else if (reg_k) {
+    rc = fgd_launch_step_reg_k(c, a, dense2, g2, d2, g1, st, &grid);
   } else if (reg_odd) {
     rc = dispatch_small_k(K, [&]<int KTc>() -> int {
       const int64_t ntiles = (c->P + (int64_t)kBlock * 4 - 1) / ((int64_t)kBlock * 4);
@@ -480,7 +498,7 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
   if ((K == 32 || K == 64) && pick_vec(4, c->P, c->ld, {theta}) == 4) {   // see consensus_split_kernel
     auto launch = [&](auto kern, int64_t ntiles) -> int {
       if (int r = persistent_grid(c, kern, kSplitBlock, 0, ntiles, &grid)) return r;
-      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld, cd_sumsq, c->done);
+      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld, cd_sumsq, c->done, K);
       return check_launch(c, "consensus_split_kernel");
     };
     const int64_t cols = 4 * kSplitBlock / (K / 16);           // columns per tile
@@ -489,6 +507,18 @@ int fgd_consensus_distance(fgd_ctx* c, const float* theta, double* cd_sumsq, voi
                         : launch(consensus_split_kernel<32, 2, 4, kSplitBlock>, ntiles))
       return r;
     return FGD_OK;
+  }
+  if (K > 16 && K < 64 && pick_vec(4, c->P, c->ld, {theta}) == 4) {        // 17-31 and 33-63 workers: zero-padded split kernels
+    const int KP = K < 32 ? 32 : 64;                                       // (run-time K before: 1.3-3.7 TB/s)
+    const int64_t cols = 4 * kSplitBlock / (KP / 16);
+    const int64_t ntiles = (c->P + cols - 1) / cols;
+    auto launch = [&](auto kern) -> int {
+      if (int r = persistent_grid(c, kern, kSplitBlock, 0, ntiles, &grid)) return r;
+      kern<<<grid, kSplitBlock, 0, st>>>(theta, c->partials, c->P, c->ld, cd_sumsq, c->done, K);
+      return check_launch(c, "consensus_split_kernel");
+    };
+    return KP == 64 ? launch(consensus_split_kernel<64, 4, 4, kSplitBlock, true>)
+                    : launch(consensus_split_kernel<32, 2, 4, kSplitBlock, true>);
   }
   if (small_odd_k(K) && pick_vec(4, c->P, c->ld, {theta}) == 4) {   // compile-time kernels for 3, 5-7, 9-15 workers
     return dispatch_small_k(K, [&]<int KTc>() -> int {

@@ -644,10 +644,14 @@ consensus_kernel(const float* __restrict__ theta, double* __restrict__ partials,
 // share a column group, each owning R = K / SPLIT rows -- the register picture of the K = 16 kernel
 // -- and exchange only their partial column sums through shared memory (double-buffered by tile
 // parity: one barrier per tile).
-template <int KT, int SPLIT, int VEC, int BLOCK>
+// PAD: the real worker count KR < KT is a run-time value (17..31 on the 32-worker shape, 33..63 on the
+// 64-worker one): rows at or beyond KR are never loaded (they count as zeros in the column sum, which is
+// divided by KR) and their sums are dropped.
+template <int KT, int SPLIT, int VEC, int BLOCK, bool PAD = false>
 __global__ void __launch_bounds__(BLOCK)
 consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ partials, int64_t P, int64_t ld,
-                       double* __restrict__ out, unsigned int* done) {
+                       double* __restrict__ out, unsigned int* done, int k_real = KT) {
+  const int KR = PAD ? k_real : KT;
   constexpr int R = KT / SPLIT;      // rows per thread
   constexpr int G = BLOCK / SPLIT;   // column groups per tile
   static_assert(KT % SPLIT == 0 && G % 32 == 0, "parts must be whole warps");
@@ -657,7 +661,7 @@ consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ par
   float sacc[R];
 #pragma unroll
   for (int m = 0; m < R; ++m) sacc[m] = 0.f;
-  const float invK = 1.0f / (float)KT;
+  const float invK = 1.0f / (float)KR;
   const int64_t ntiles = (P + (int64_t)G * VEC - 1) / ((int64_t)G * VEC);
   int it = 0;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
@@ -667,7 +671,10 @@ consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ par
     Pack<VEC> sum = p_zero<VEC>();
     if (live) {
 #pragma unroll
-      for (int m = 0; m < R; ++m) t[m] = ld_stream<VEC>(theta + (size_t)(r0 + m) * ld + col);
+      for (int m = 0; m < R; ++m) {
+        if (!PAD || r0 + m < KR) t[m] = ld_stream<VEC>(theta + (size_t)(r0 + m) * ld + col);
+        else t[m] = p_zero<VEC>();
+      }
 #pragma unroll
       for (int m = 0; m < R; ++m) sum = p_add<VEC>(sum, t[m]);
     }
@@ -699,14 +706,14 @@ consensus_split_kernel(const float* __restrict__ theta, double* __restrict__ par
     if (lane == 0) red[warp][m] = d;
   }
   __syncthreads();
-  if (tid < KT) {                    // worker tid = rows of part tid / R, summed over that part's warps
+  if (tid < KR) {                    // worker tid = rows of part tid / R, summed over that part's warps
     const int q = tid / R, j = tid % R;
     double d = 0.0;
 #pragma unroll
     for (int w = 0; w < G / 32; ++w) d += red[q * (G / 32) + w][j];
-    partials[(size_t)blockIdx.x * KT + tid] = d;
+    partials[(size_t)blockIdx.x * KR + tid] = d;
   }
-  finalize_in_last_cta(partials, KT, out, done);
+  finalize_in_last_cta(partials, KR, out, done);
 }
 
 // Global average with many workers, same split: out = column mean as one row (out_is_vector) or

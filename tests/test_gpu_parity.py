@@ -58,6 +58,10 @@ MIX_CASES = [
     (48, 9001, ("ring",)), (40, 5000, ("dense", gen.sinkhorn_W(8, 40))), (33, 4100, ("matching",)), (63, 3000, ("mean",)),
     (32, 6002, ("dense", gen.sinkhorn_W(7, 32))), (24, 7000, ("ring", 0.3)), (17, 2000, ("dense", gen.sinkhorn_W(9, 17))),
     (64, 20000, ("hypercube", 0.1)), (8, 30000, ("hypercube", 0.2)), (16, 9000, ("randgraph", 5, 0.2)), (40, 3000, ("randgraph", 3)), (7, 2000, ("randgraph", 2)),
+    # sparse mixes above 16 workers: the TMA-pipelined row gather (run-time worker and slot counts, ragged tails)
+    (17, 1001, ("ring",)), (23, 70003, ("matching",)), (31, 5000, ("circulant", 2)), (32, 9999, ("circulant", 3, 0.2)),
+    (47, 3000, ("randgraph", 8)), (57, 130, ("ring", 0.3)), (63, 20001, ("randgraph", 5, 0.2)), (64, 127, ("matching",)),
+    (20, 4096, ("identity",)),
     # every worker count up to 16 that is not a power of two has stand-alone kernels of its own
     (3, 5001, ("ring",)), (6, 4100, ("matching",)), (6, 70001, ("ring", 0.2)), (7, 9000, ("ring",)), (10, 6000, ("randgraph", 3)),
     (11, 3001, ("ring", 0.3, fgd.FGD_RENORM_SELF_ABSORB)), (12, 8000, ("matching",)), (13, 5000, ("randgraph", 5)),

@@ -117,6 +117,28 @@ def test_tensor_core_mix_wait_runs_out_and_context_recovers():
     assert torch.equal(out, out_f) and bool((out != 0).any())
 
 
+def test_gather_mix_wait_runs_out_and_context_recovers():
+    """The stand-alone sparse mix above 16 workers (TMA-pipelined row gather, run-time worker count)."""
+    K, P = 40, 148 * 4 * 4 * 128 + 36          # more tiles than stages for every CTA at four CTAs per SM
+    W = fgd.MixDesc.ring(K)
+    th0, _, _ = _inputs(K, P, 34)
+    ctx = fgd.Context(K, P)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SPIN_LIMIT, SPIN)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SKIP_TILE, 2)
+    out = torch.zeros_like(th0)
+    fgd.fgd_mix(ctx, W, th0, out)
+    _expect_timeout_once(ctx)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SPIN_LIMIT, 0)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SKIP_TILE, -1)
+    out.zero_()
+    fgd.fgd_mix(ctx, W, th0, out)
+    fgd.fgd_device_status(ctx)
+    fresh, out_f = fgd.Context(K, P), torch.zeros_like(th0)
+    fgd.fgd_mix(fresh, W, th0, out_f)
+    fgd.fgd_device_status(fresh)
+    assert torch.equal(out, out_f) and bool((out != 0).any())
+
+
 def test_debug_set_rejects_unknown_keys():
     ctx = fgd.Context(4, 1024)
     with pytest.raises(fgd.FgdError) as e:
