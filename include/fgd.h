@@ -109,10 +109,11 @@ int64_t fgd_launch_count(const fgd_ctx* ctx);
  *   FGD_DEBUG_SKIP_TILE   every CTA of the TMA-pipelined kernels (fused step, tensor-core step,
  *                         tensor-core mix) announces but never issues the loads of its value-th
  *                         tile (0-based), so the wait for that tile runs out; -1 = off (default).
- *   FGD_DEBUG_GOSSIP_PATH how the tensor-core step (more than 48 workers) computes a sparse Mix1 that is
- *                         fused into it: 0 = by neighbour-slot count (default), 1 = gathered from the
- *                         staged theta_prev, 2 = as a second group of MMAs.  For tests and measurements
- *                         that need either kernel whatever the slot count; results agree to rounding.
+ *   FGD_DEBUG_GOSSIP_PATH which kernel takes a step above 16 workers: 0 = the measured choice (default);
+ *                         1 / 2 = the tensor-core kernel, a fused sparse Mix1 gathered from the staged
+ *                         theta_prev (1) or, above 48 workers, run as a second group of MMAs (2); 3 = the
+ *                         row-gather kernel (sparse Mix2 only).  For tests and measurements that need one
+ *                         kernel whatever the shape; results agree to rounding.
  * All stay set until changed.  Not for production use. */
 typedef enum { FGD_DEBUG_SPIN_LIMIT = 1, FGD_DEBUG_SKIP_TILE = 2, FGD_DEBUG_GOSSIP_PATH = 3 } fgd_debug_key;
 int fgd_debug_set(fgd_ctx* ctx, int key, int64_t value);

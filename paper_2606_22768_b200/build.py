@@ -16,7 +16,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfgd.so")
 SOURCES = ["fgd_api.cu", "fgd_step_tma.cu", "fgd_step_tma_g0.cu", "fgd_step_tma_g1.cu", "fgd_step_tma_g2.cu", "fgd_step_tma_g3.cu",
-           "fgd_step_reg.cu", "fgd_mix_gather_tma.cu", "fgd_noalloc.cu", "fgd_js.cu", "fgd_pattern_probe.cu", "fgd_from_host.cu", "fgd_host.cpp"]
+           "fgd_step_reg.cu", "fgd_step_rows.cu", "fgd_mix_gather_tma.cu", "fgd_noalloc.cu", "fgd_js.cu", "fgd_pattern_probe.cu", "fgd_from_host.cu", "fgd_host.cpp"]
 HEADERS = ["fgd_kernels.cuh", "fgd_step_tma.cuh", "fgd_step_dense_tc.cuh", "fgd_mix_dense_tc.cuh", "fgd_step_gossip_tc.cuh", "fgd_step_tma.h", "fgd_tma_host.h", "fgd_step_tma_launch.inl", "fgd_ctx.h", "fgd_internal.h", "fgd_nvtx.h", os.path.join(ROOT, "include", "fgd.h")]
 
 NVCC_FLAGS = ["-std=c++20", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

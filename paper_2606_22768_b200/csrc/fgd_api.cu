@@ -111,7 +111,7 @@ int fgd_debug_set(fgd_ctx* c, int key, int64_t value) {
       c->dbg_skip_tile = (int)value;
       return FGD_OK;
     case FGD_DEBUG_GOSSIP_PATH:
-      if (value < 0 || value > 2) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: gossip path %lld out of range", (long long)value);
+      if (value < 0 || value > 3) return fail(c, FGD_ERR_INVALID_ARG, "fgd_debug_set: gossip path %lld out of range", (long long)value);
       c->dbg_gossip_path = (int)value;
       return FGD_OK;
     default:
@@ -417,12 +417,18 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
       for (int m = 0; m < K; ++m)
         for (int n = 0; n < K; ++n) d2.Wt[n * K + m] = (float)Wd[m * K + n];
   }
-  if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma))
+  const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
+  const bool can_rows = K > 16 && fgd_step_rows_eligible(c, a, dense2, g2);
+  // A sparse Mix1 fused above 32 workers: the row gather (TB/s rows / tensor-core kernel; ring + ring K = 33 5.7/3.7,
+  // 40 6.1/4.2, 48 6.2/4.7, 56 5.8/4.2, 64 5.7/4.8; matching 5.6-6.2/3.7-4.9; four slots 4.6-5.2/3.2-4.7), except five
+  // and more slots in BOTH mixes from 49 workers, where both mixes as MMAs cost the same whatever the slot count
+  // (K = 64, six slots: 4.1/4.8).  At 32 workers and below the two-group tensor-core kernel or a register kernel wins.
+  const bool rows_auto = gossip1 && K >= 33 && !(K >= 49 && g1.D >= 5 && g2.D >= 5);
+  if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma && !can_rows))
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");
   const bool reg_odd = small_odd_k(K) && pick_vec(4, c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next}) == 4;
   const bool reg_k = fgd_reg_k_built(K) && pick_vec(2, c->P, c->ld, {theta_local, theta_prev, momentum, theta_new, x, a.x_next}) == 2;
-  const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
   // 17-31 workers: the register kernel compiled for that count against the tensor-core kernel zero-padded to
   // 32 (measured, TB/s register / tensor cores, K = 17 | 20 | 24 | 28): ring 6.0/5.2 | 6.0/5.9 | 5.6/5.7 | 5.7/5.6;
   // four slots 5.9/4.9 | 5.8/4.9 | 4.8/5.8 | 5.0/5.5; matrix x 4.3/3.1 | 4.3/3.6 | 3.5/4.3 | 3.4/5.0; ring + ring fused
@@ -432,7 +438,11 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
                           (K <= 20 || (gossip1 && ((gslots <= 1 && K <= 25) || (gslots <= 2 && K <= 21))));
   const bool reg_odd_auto = reg_odd && reg_beats_pipelined(K, dense2, a.xsrc == XSRC_MATRIX, gossip1,
                                                            dense2 ? 0 : g2.D, gossip1 ? g1.D : 0);
-  if (can_tc && c->path != FGD_PATH_REGISTER && !reg_k_auto) {
+  if (can_rows && (c->dbg_gossip_path == 3 ||
+                   (c->dbg_gossip_path == 0 && ((c->path == FGD_PATH_TMA_FP32 && (!can_tma || KT == 0)) ||
+                                                (c->path == FGD_PATH_AUTO && rows_auto))))) {
+    rc = fgd_launch_step_rows(c, a, g2, g1, st, &grid);
+  } else if (can_tc && c->path != FGD_PATH_REGISTER && !reg_k_auto) {
     rc = fgd_launch_step_dense_tc(c, a, d2, g1, st, &grid);
   } else if (can_tma && c->path != FGD_PATH_REGISTER && !reg_k_auto &&
              !(c->path == FGD_PATH_AUTO && (K <= 2 || (dense2 && (KT == 8 || KT == 16)) || reg_odd_auto))) {

@@ -36,7 +36,7 @@ struct fgd_ctx {
   int64_t launches = 0;
   uint32_t dbg_spin_limit = 0;   // fgd_debug_set: polls before a device-side wait gives up (0 = the default)
   int dbg_skip_tile = -1;        // fgd_debug_set: tile whose loads the pipelined kernels withhold (-1 = none)
-  int dbg_gossip_path = 0;       // fgd_debug_set: 0 = by slot count, 1 = gather, 2 = MMAs (tensor-core step, sparse Mix1 fused)
+  int dbg_gossip_path = 0;       // fgd_debug_set: 0 = measured choice, 1 = tensor-core gather, 2 = tensor-core MMAs, 3 = row-gather kernel
   char err[256] = "";
   std::map<std::pair<const void*, size_t>, int> occupancy;  // (kernel, smem) -> CTAs per SM
   // fgd_outer_step_from_host only (created by its first call): copy stream, one event per column

@@ -26,6 +26,10 @@ int fgd_launch_step_dense_tc(fgd_ctx* c, const fgd::StepArgs& a, const fgd::Dens
 // Stand-alone sparse mix as a TMA-pipelined row gather, any worker and slot count (fgd_mix_gather_tma.cu).
 bool fgd_mix_gather_tma_eligible(const fgd_ctx* c, const float* in, const float* out);
 int fgd_launch_mix_gather_tma(fgd_ctx* c, const float* in, float* out, const fgd::GatherMix& gm, cudaStream_t st);
+// Fused step with a sparse Mix2 as a TMA-pipelined row gather, any worker and slot count (fgd_step_rows.cu).
+bool fgd_step_rows_eligible(const fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g2);
+int fgd_launch_step_rows(fgd_ctx* c, const fgd::StepArgs& a, const fgd::GatherMix& g2, const fgd::GatherMix& g1,
+                         cudaStream_t st, int* grid_out);
 // Register-path fused step compiled for the worker counts 17..31 (fgd_step_reg.cu; two columns per thread).
 bool fgd_reg_k_built(int K);
 int fgd_launch_step_reg_k(fgd_ctx* c, const fgd::StepArgs& a, bool dense2, const fgd::GatherMix& g2, const fgd::DenseMix& d2,

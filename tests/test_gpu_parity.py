@@ -16,8 +16,8 @@ from tests.gpu_util import (Scenario, assert_cd_close, assert_param_close, check
 pytestmark = pytest.mark.gpu
 
 SINK64 = gen.sinkhorn_W(0, 64)
-PATHS = [pytest.param(fgd.FGD_PATH_TMA, id="tma"), pytest.param(fgd.FGD_PATH_REGISTER, id="reg"),
-         pytest.param(fgd.FGD_PATH_TMA_FP32, id="tma_fp32")]
+PATHS = [pytest.param(fgd.FGD_PATH_AUTO, id="auto"), pytest.param(fgd.FGD_PATH_TMA, id="tma"),
+         pytest.param(fgd.FGD_PATH_REGISTER, id="reg"), pytest.param(fgd.FGD_PATH_TMA_FP32, id="tma_fp32")]
 
 
 def _inputs(K, P, seed=0, worker_std=5e-4, sigma=1e-3):

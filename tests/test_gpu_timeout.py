@@ -78,7 +78,26 @@ def test_gossip_tensor_core_step_wait_runs_out_and_context_recovers():
         fgd.fgd_outer_step(ctx, m2, m1, None, False, loc0, th, mom, th, 0.7, 0.9, cd)
         return cd
 
+    _gossip_timeout_case(K, P, run, th0, mom0, gossip_path=2)
+
+
+def test_row_gather_step_wait_runs_out_and_context_recovers():
+    """The step with a sparse Mix1 fused above 32 workers (TMA-pipelined row gather, run-time worker count)."""
+    K, P = 40, 148 * 4 * 128 + 36
+    m1, m2 = fgd.MixDesc.ring(K), fgd.MixDesc.ring(K)
+    th0, loc0, mom0 = _inputs(K, P, 35)
+
+    def run(ctx, th, mom):
+        cd = torch.zeros(K, dtype=torch.float64, device="cuda")
+        fgd.fgd_outer_step(ctx, m2, m1, None, False, loc0, th, mom, th, 0.7, 0.9, cd)
+        return cd
+
+    _gossip_timeout_case(K, P, run, th0, mom0, gossip_path=3)
+
+
+def _gossip_timeout_case(K, P, run, th0, mom0, gossip_path):
     ctx = fgd.Context(K, P)
+    fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_GOSSIP_PATH, gossip_path)
     fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SPIN_LIMIT, SPIN)
     fgd.fgd_debug_set(ctx, fgd.FGD_DEBUG_SKIP_TILE, 1)
     run(ctx, th0.clone(), mom0.clone())
@@ -89,6 +108,7 @@ def test_gossip_tensor_core_step_wait_runs_out_and_context_recovers():
     cd = run(ctx, th, mom)
     fgd.fgd_device_status(ctx)
     fresh = fgd.Context(K, P)
+    fgd.fgd_debug_set(fresh, fgd.FGD_DEBUG_GOSSIP_PATH, gossip_path)
     th_f, mom_f = th0.clone(), mom0.clone()
     cd_f = run(fresh, th_f, mom_f)
     fgd.fgd_device_status(fresh)
