@@ -419,15 +419,16 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   }
   const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
   const bool can_rows = K > 16 && fgd_step_rows_eligible(c, a, dense2, g2);
-  // A sparse Mix1 fused above 32 workers: the row gather (TB/s rows / tensor-core kernel; ring + ring K = 33 5.7/3.7,
-  // 40 6.1/4.2, 48 6.2/4.7, 56 5.8/4.2, 64 5.7/4.8; matching 5.6-6.2/3.7-4.9; four slots 4.6-5.2/3.2-4.7), except five
-  // and more slots in BOTH mixes from 49 workers, where both mixes as MMAs cost the same whatever the slot count
-  // (K = 64, six slots: 4.1/4.8).  At 32 workers and below the two-group tensor-core kernel or a register kernel wins.
-  // A matrix-valued x (prefetched one tile ahead by the rows' owners) likewise: ring Mix2 K = 33 5.5/4.3, 40 5.8/4.8,
-  // 48 6.2/5.9, 56 5.9/4.5, 64 6.4/5.0 (four slots 5.0-6.2/4.2-5.6); with up to two slots also at 21-31 workers (4.4-5.1/3.8-4.9).
-  // x one value per column stays on the tensor-core kernel (within 3 % of each other from 33 workers, behind it below).
-  const bool rows_auto = (gossip1 && K >= 33 && !(K >= 49 && g1.D >= 5 && g2.D >= 5)) ||
-                         (a.xsrc == XSRC_MATRIX && (K >= 33 || (K >= 21 && K <= 31 && g2.D <= 2)));
+  // The row gather (fgd_step_rows.cu) takes a sparse Mix1 fused into the step and a matrix-valued x at 17-28 and
+  // at 33-64 workers (TB/s rows / best other kernel; ring + ring fused K = 17 5.5/5.4, 21 5.9/4.6, 24 5.8/4.6,
+  // 28 5.6/5.2, 33 5.7/3.7, 40 6.1/4.2, 48 6.2/4.7, 56 5.8/4.2, 64 5.7/4.8; matching fused 5.6-6.2/3.7-5.9; four slots
+  // 4.6-5.4/3.2-4.7; ring Mix2 with a matrix x K = 17 6.3/4.3, 24 6.1/4.3, 33 5.5/4.3, 48 6.2/5.9, 64 6.4/5.0).  Not
+  // with five and more slots in BOTH mixes from 25 workers, where the tensor-core kernels (Mix2, from 49 workers
+  // also Mix1, as MMAs whatever the slot count) are ahead (K = 64, six slots: 4.1/4.8); not at 29-32 workers, where
+  // its one CTA per SM shows and the two-group tensor-core kernel wins (K = 31: 4.6/6.0).  x one value per column
+  // stays where it was: the two are within 4 % of each other.
+  const bool rows_auto = (gossip1 || a.xsrc == XSRC_MATRIX) && (K <= 28 || K >= 33) &&
+                         !(gossip1 && K >= 25 && g1.D >= 5 && g2.D >= 5);
   if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma && !can_rows))
     return fail(c, FGD_ERR_UNSUPPORTED,
                 "fgd_outer_step: the TMA path needs 16-byte aligned tensors, ld %% 4 == 0 and room for two stages");

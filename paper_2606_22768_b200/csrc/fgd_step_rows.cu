@@ -23,7 +23,6 @@ using namespace fgd;
 namespace {
 
 constexpr int kRowWarps = 8, kRowConsumers = 32 * kRowWarps, kRowCols = 128, kRowMaxStages = 6;
-constexpr int kRowsPerWarp = FGD_MAX_K / kRowWarps;          // 8
 constexpr int kRowF4 = kRowCols / 4;                         // float4 per staged row
 constexpr size_t kRowStatic = 26 * 1024;                     // static shared memory: tables, exchange rows, barriers (25.2 KB)
 
@@ -69,8 +68,11 @@ __device__ __forceinline__ void st_cols(float* p, const float4 v, int64_t col, i
 
 // D2T / D1T: neighbour slots of Mix2 / of a fused gossip Mix1 as unrolled (1, 2, 4 or 8 >= the used
 // count; unused slots point at the row itself with weight 0).  D1T = 0: Mix1 is not a gossip mix.
-template <int D2T, int D1T>
-__global__ void __launch_bounds__(kRowConsumers + 32, 1)
+// RPW: rows per warp, 8 (any worker count, one CTA per SM) or 4 (up to 32 workers: half the registers, so
+// that two CTAs share an SM where two of their two-stage rings fit -- with few rows a tile is short and its
+// fixed chain of waits, one CTA's worth, would otherwise show).
+template <int D2T, int D1T, int RPW>
+__global__ void __launch_bounds__(kRowConsumers + 32, RPW == 4 ? 2 : 1)
 outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix m1,
                        const __grid_constant__ CUtensorMap tm_prev, const __grid_constant__ CUtensorMap tm_local,
                        const __grid_constant__ CUtensorMap tm_mom) {
@@ -112,9 +114,9 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
   }
   __syncthreads();
 
-  double dacc[kRowsPerWarp];                       // consensus sums of rows warp, warp + 8, ... (this lane's columns)
+  double dacc[RPW];                       // consensus sums of rows warp, warp + 8, ... (this lane's columns)
 #pragma unroll
-  for (int r = 0; r < kRowsPerWarp; ++r) dacc[r] = 0.0;
+  for (int r = 0; r < RPW; ++r) dacc[r] = 0.0;
 
   if (warp == kRowWarps) {
     // ===================================================== producer warp (one elected lane)
@@ -156,7 +158,7 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
     const bool has_barrier = need_mean || x_mean || PRE;
     // x from global memory (a vector or a matrix) is fetched one tile ahead into registers: its latency
     // would otherwise stand at the head of every tile (x per column: 4.5 -> 5.7 TB/s at 33 workers)
-    float4 xv_next = make_float4(0.f, 0.f, 0.f, 0.f), xm_next[kRowsPerWarp];
+    float4 xv_next = make_float4(0.f, 0.f, 0.f, 0.f), xm_next[RPW];
     auto fetch_x = [&](int64_t tile_) {
       const int64_t c_ = tile_ * kRowCols + 4 * lane;
       if (tile_ >= ntiles || c_ >= P) return;
@@ -164,19 +166,19 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
       if (x_vector) xv_next = ld_cols(a.x + c_, c_, P, whole_);
       if (x_matrix) {
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r)
+        for (int r = 0; r < RPW; ++r)
           if (warp + kRowWarps * r < K) xm_next[r] = ld_cols(a.x + (size_t)(warp + kRowWarps * r) * ld + c_, c_, P, whole_);
       }
     };
 #pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) xm_next[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r = 0; r < RPW; ++r) xm_next[r] = make_float4(0.f, 0.f, 0.f, 0.f);
     fetch_x(blockIdx.x);
     int64_t i = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++i) {
       const int s = (int)(i % STAGES), par = (int)(i & 1);
-      float4 xc = xv_next, xm[kRowsPerWarp];         // x when it is one value per column / this warp's rows of a matrix x
+      float4 xc = xv_next, xm[RPW];         // x when it is one value per column / this warp's rows of a matrix x
 #pragma unroll
-      for (int r = 0; r < kRowsPerWarp; ++r) xm[r] = xm_next[r];
+      for (int r = 0; r < RPW; ++r) xm[r] = xm_next[r];
       fetch_x(tile + gridDim.x);
       const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars[s]), (uint32_t)(i / STAGES) & 1, ta.spin_limit));
       if (!ok) {                                     // (taken per warp; the CTA-wide decision follows the barrier)
@@ -208,10 +210,10 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
         rows_bar_sync(3, kRowConsumers);
         if (*(volatile int*)&abort_flag) break;      // uniform: written before the barrier
       }
-      float4 tn[kRowsPerWarp];
+      float4 tn[RPW];
       float4 colsum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int r = 0; r < kRowsPerWarp; ++r) {
+      for (int r = 0; r < RPW; ++r) {
         const int m = warp + kRowWarps * r;
         tn[r] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (m < K && ok) {
@@ -258,7 +260,7 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
         if (a.x_next != nullptr && warp == 0 && any) st_cols(a.x_next + col, mean, col, P, whole);
         if (want_cd) {
 #pragma unroll
-          for (int r = 0; r < kRowsPerWarp; ++r) {
+          for (int r = 0; r < RPW; ++r) {
             if (warp + kRowWarps * r < K) {
               const float4 d = f4_sub(tn[r], mean);
               dacc[r] += (double)fmaf(d.x, d.x, fmaf(d.y, d.y, fmaf(d.z, d.z, d.w * d.w)));
@@ -274,7 +276,7 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
   // ---- consensus sums: every row belongs to one warp, so a warp-level reduction finishes it
   if (want_cd && warp < kRowWarps) {
 #pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) {
+    for (int r = 0; r < RPW; ++r) {
       const int m = warp + kRowWarps * r;
       double d = dacc[r];
 #pragma unroll
@@ -309,8 +311,10 @@ int fgd_launch_step_rows(fgd_ctx* c, const StepArgs& a, const GatherMix& g2, con
   if (int rc = make_tensor_map(c, &tl, a.theta_local, kRowCols)) return rc;
   if (int rc = make_tensor_map(c, &tm, a.momentum, kRowCols)) return rc;
   const size_t stage = 3 * (size_t)c->K * kRowCols * 4;
-  // one CTA per SM (registers): as many stages as its shared memory holds
-  int stages = (int)(((size_t)c->max_smem_optin - kRowStatic - 128) / stage);
+  // one CTA per SM: as many stages as its shared memory holds; up to 28 workers two CTAs with two or three stages each
+  const bool two_ctas = c->K <= 28;
+  const size_t budget = two_ctas ? (size_t)c->max_smem_optin / 2 - 2048 : (size_t)c->max_smem_optin;
+  int stages = (int)((budget - kRowStatic - 128) / stage);
   stages = stages < 2 ? 2 : (stages > kRowMaxStages ? kRowMaxStages : stages);
   const size_t smem = 128 + stages * stage;
   TmaStepArgs ta;
@@ -329,7 +333,7 @@ int fgd_launch_step_rows(fgd_ctx* c, const StepArgs& a, const GatherMix& g2, con
   const bool gossip1 = a.xsrc == XSRC_FUSED && g1.kind == KMIX_GATHER;
   const int d2 = slot_class(g2.D), d1 = gossip1 ? slot_class(g1.D) : 0;
 #define FGD_CASE(x2, x1) \
-  if (d2 == x2 && d1 == x1) return launch(outer_step_rows_kernel<x2, x1>);
+  if (d2 == x2 && d1 == x1) return two_ctas ? launch(outer_step_rows_kernel<x2, x1, 4>) : launch(outer_step_rows_kernel<x2, x1, 8>);
   FGD_CASE(1, 0) FGD_CASE(2, 0) FGD_CASE(4, 0) FGD_CASE(8, 0)
   FGD_CASE(1, 1) FGD_CASE(2, 1) FGD_CASE(4, 1) FGD_CASE(8, 1)
   FGD_CASE(1, 2) FGD_CASE(2, 2) FGD_CASE(4, 2) FGD_CASE(8, 2)
