@@ -80,6 +80,7 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the round: the fused step across worker counts and mix kinds (4 GB per tensor)")
     ap.add_argument("--sweep-ks", default="", help="with --sweep: comma-separated worker counts (default: the full list)")
+    ap.add_argument("--sweep-bytes", type=int, default=4_000_000_000, help="with --sweep: bytes per [K,P] tensor (smaller for an ncu capture)")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
@@ -499,7 +500,8 @@ def run_ours(args):
     if args.sweep:
         if rank == 0:
             ks = tuple(int(k) for k in args.sweep_ks.split(",")) if args.sweep_ks else None
-            print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak(), **({"Ks": ks} if ks else {}))), flush=True)
+            print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak(), tensor_bytes=args.sweep_bytes,
+                                         **({"Ks": ks} if ks else {}))), flush=True)
         return
     cfg = dict(CONFIGS[args.config])
     if args.cols:
