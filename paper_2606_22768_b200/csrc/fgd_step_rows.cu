@@ -161,7 +161,12 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
     float4 xv_next = make_float4(0.f, 0.f, 0.f, 0.f), xm_next[RPW];
     auto fetch_x = [&](int64_t tile_) {
       const int64_t c_ = tile_ * kRowCols + 4 * lane;
-      if (tile_ >= ntiles || c_ >= P) return;
+      if (tile_ >= ntiles || c_ >= P) {              // columns outside the tensor count as zeros everywhere below
+        xv_next = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int r = 0; r < RPW; ++r) xm_next[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+      }
       const bool whole_ = c_ + 3 < P;
       if (x_vector) xv_next = ld_cols(a.x + c_, c_, P, whole_);
       if (x_matrix) {

@@ -154,12 +154,14 @@ def test_more_than_2_to_31_columns():
 
 
 @pytest.mark.parametrize("K,P,mix1,fused", [(40, 40_000_037, ("mean",), False),      # padded to 48 workers, ragged tail
-                                            (56, 30_000_004, ("ring", 0.1), True),   # padded to 64, gossip Mix1 fused
+                                            (56, 30_000_004, ("ring", 0.1), True),   # row gather, gossip Mix1 fused (56 rows, nothing padded)
                                             (12, 100_000_002, ("ring",), False),     # compile-time 12, matrix-valued x
                                             (13, 70_000_004, ("mean",), False),      # zero-padded onto the 16-worker fp32 kernel
                                             (10, 50_000_002, ("ring", 0.1), True),   # zero-padded onto 12, gossip Mix1 fused
-                                            (64, 20_000_003, ("ring", 0.1), True),   # gossip Mix1 gathered at 64 workers, ragged tail
-                                            (64, 20_000_003, ("hypercube", 0.1), True)])  # both mixes as MMAs, ragged tail
+                                            (64, 20_000_003, ("ring", 0.1), True),   # row gather with the gossip Mix1 fused, ragged tail
+                                            (64, 20_000_003, ("hypercube", 0.1), True),   # both mixes as MMAs, ragged tail
+                                            (24, 60_000_002, ("ring", 0.1), False),       # row gather, matrix-valued x, two CTAs per SM, ragged tail
+                                            (48, 30_000_001, ("matching", 0.1), False)])  # row gather, matrix-valued x, one CTA per SM
 def test_full_size_other_worker_counts(K, P, mix1, fused):
     """Worker counts beside the benchmark configurations at sizes of many thousand tiles per CTA:
     zero-padded tensor-core shapes and the 12-worker kernel, 3 free-running rounds, sampled blocks."""

@@ -183,6 +183,16 @@ STEP_CASES = [
     (8, 5001, ("mean",), ("hypercube", 0.3)),
     (32, 7000, ("hypercube",), ("hypercube", 0.1)),
     (32, 4001, ("mean",), ("hypercube",)),
+    # the row-gather kernel (fused gossip Mix1 or matrix x at 17-28 and 33-64 workers): fewer columns than a tile,
+    # ragged tails, one to eight neighbour slots, both CTA shapes
+    (40, 3, ("ring",), ("ring",)),
+    (24, 130, ("matching",), ("ring", 0.3)),
+    (64, 127, ("ring",), ("circulant", 2)),
+    (28, 4100, ("randgraph", 3), ("randgraph", 5)),
+    (33, 5000, ("circulant", 4, 0.2), ("circulant", 4)),
+    (21, 9001, ("identity",), ("ring",)),
+    (17, 70002, ("matching", 0.2), ("matching",)),
+    (63, 8000, ("randgraph", 8, 0.1), ("ring",)),
     # fewer columns than one tile (and than one vector)
     (64, 5, ("mean",), ("dense", SINK64)),
     (48, 1, ("mean",), ("ring",)),
