@@ -105,7 +105,10 @@ def test_mix_mean_vector_output(K, P):
                                      (5, 7777, 7780), (1, 50, 50), (2, 3, 4), (64, 150004, 150016), (32, 200000, 200000),
                                      (64, 131, 132), (32, 4, 4)]
                          + [(K, 20000 + 37 * K, 20000 + 37 * K + (4 - (37 * K) % 4) % 4) for K in (3, 6, 7, 9, 10, 11, 12, 13, 14, 15)]
-                         + [(13, 5001, 5001)])      # odd row stride: the run-time-K kernel
+                         + [(13, 5001, 5001)]       # odd row stride: the run-time-K kernel
+                         # 17-31 / 33-63 workers on the 32- / 64-worker split kernels with the rows beyond K left out
+                         + [(17, 30001, 30004), (24, 4096, 4096), (31, 70003, 70004), (33, 20002, 20004), (47, 9000, 9000),
+                            (56, 131, 132), (63, 50001, 50004), (40, 3, 4), (23, 20001, 20001)])
 def test_consensus_distance(K, P, ld):
     ld = P if ld is None else ld
     th = gen.theta0(5, K, P, 0.02, 7e-4)
