@@ -33,7 +33,12 @@
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
  *    stream): tensors must stay alive until the stream reaches that point.
  *  - Fast path: base pointers 16-byte aligned and ld % 4 == 0; otherwise an element-wise
- *    path is used (slower, not an error).
+ *    path is used (slower, not an error).  FULL speed needs rows that start on 128-byte
+ *    boundaries (128-byte aligned bases, ld % 32 == 0): every kernel moves 512-byte to 4-KB row
+ *    segments, and a segment that starts inside a 32-byte DRAM sector leaves partly written
+ *    sectors at both ends.  Measured on the fused step (4 GB per tensor): ld % 32 == 0 -> 1.00;
+ *    ld % 8 == 0 only -> 0.97 (8 and 16 workers) to 0.90 (64 workers); ld % 4 == 0 only -> 0.91
+ *    (16 workers) to 0.65-0.70 (40 and 64 workers).  The caller owns the layout: pad ld.
  *  - Deterministic: the same inputs give bit-identical outputs (no floating-point atomics).
  *  - Threads: a context is NOT re-entrant.  It carries the last error string, an occupancy cache
  *    and (during fgd_outer_step_from_host) a temporarily narrowed column count, so one context
