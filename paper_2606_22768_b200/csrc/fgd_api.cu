@@ -422,12 +422,15 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   // The row gather (fgd_step_rows.cu) takes a sparse Mix1 fused into the step and a matrix-valued x at 17-28 and
   // at 33-64 workers (TB/s rows / best other kernel; ring + ring fused K = 17 5.5/5.4, 21 5.9/4.6, 24 5.8/4.6,
   // 28 5.6/5.2, 33 5.7/3.7, 40 6.1/4.2, 48 6.2/4.7, 56 5.8/4.2, 64 5.7/4.8; matching fused 5.6-6.2/3.7-5.9; four slots
-  // 4.6-5.4/3.2-4.7; ring Mix2 with a matrix x K = 17 6.3/4.3, 24 6.1/4.3, 33 5.5/4.3, 48 6.2/5.9, 64 6.4/5.0).  Not
+  // 4.6-5.4/3.2-4.7; ring Mix2 with a matrix x K = 17 6.3/4.3, 24 6.4/4.3, 33 5.5/4.3, 40 5.5/5.2, 56 6.1/4.5; from 59
+  // workers its stages push the shared-memory carve-out to the maximum, the 28 KB of L1 left cannot hold the 30 KB
+  // of x that the rows' owners have in flight one tile ahead, and it falls to 4.8 against 5.0-5.4, so the
+  // tensor-core kernel keeps a matrix x there).  Not
   // with five and more slots in BOTH mixes from 25 workers, where the tensor-core kernels (Mix2, from 49 workers
   // also Mix1, as MMAs whatever the slot count) are ahead (K = 64, six slots: 4.1/4.8); not at 29-32 workers, where
   // its one CTA per SM shows and the two-group tensor-core kernel wins (K = 31: 4.6/6.0).  x one value per column
   // stays where it was: the two are within 4 % of each other.
-  const bool rows_auto = (gossip1 || a.xsrc == XSRC_MATRIX) && (K <= 28 || K >= 33) &&
+  const bool rows_auto = (gossip1 || (a.xsrc == XSRC_MATRIX && K <= 58)) && (K <= 28 || K >= 33) &&
                          !(gossip1 && K >= 25 && g1.D >= 5 && g2.D >= 5);
   if ((c->path == FGD_PATH_TMA && !can_tma && !can_tc) || (c->path == FGD_PATH_TMA_FP32 && !can_tma && !can_rows))
     return fail(c, FGD_ERR_UNSUPPORTED,

@@ -253,6 +253,8 @@ outer_step_rows_kernel(const TmaStepArgs ta, const GatherMix m2, const GatherMix
         }
       }
       if (need_mean) *reinterpret_cast<float4*>(&xch[par][0][warp][4 * lane]) = colsum;
+      // (the in-place g rows were written through the generic proxy; the next TMA copy into this stage is not)
+      if constexpr (PRE) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();                                  // every lane has read its part of the stage
       if (lane == 0 && ok) mbar_arrive(smem_u32(&bars[kRowMaxStages + s]));
       if (need_mean) {
