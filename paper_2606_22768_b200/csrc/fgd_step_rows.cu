@@ -49,7 +49,12 @@ __device__ __forceinline__ void f4_add(float4& acc, const float4 a) {
 }
 // Four columns starting at col of a row, zeros beyond P (whole: all four are inside).
 __device__ __forceinline__ float4 ld_cols(const float* p, int64_t col, int64_t P, bool whole) {
-  if (whole) return __ldcs(reinterpret_cast<const float4*>(p));
+  if (whole) {                                      // x is read once and never written here: past L1
+    float4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+  }
   float r[4];
 #pragma unroll
   for (int t = 0; t < 4; ++t) r[t] = col + t < P ? p[t] : 0.f;
