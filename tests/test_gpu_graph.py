@@ -18,6 +18,8 @@ pytestmark = pytest.mark.gpu
     (16, 50001, ("hypercube",), ("hypercube",), False),   # matrix-valued Mix1 result on the side stream
     (16, 30000, ("ring",), ("ring",), True),              # gossip Mix1 fused: one kernel + finalisation
     (64, 9000, ("mean",), ("dense", gen.sinkhorn_W(0, 64)), False),   # tensor-core kernel
+    (40, 20001, ("ring",), ("matching",), True),          # row-gather step (gossip Mix1 fused, run-time worker count)
+    (24, 7000, ("ring",), ("ring",), False),              # row-gather mix on the side stream + row-gather step with a matrix x
 ])
 def test_round_replayed_from_a_cuda_graph(K, P, mix1, mix2, fused):
     seed = 5
