@@ -422,9 +422,9 @@ int fgd_outer_step_ex(fgd_ctx* c, const fgd_mix_desc* mix2, const fgd_mix_desc* 
   // The row gather (fgd_step_rows.cu) takes a sparse Mix1 fused into the step and a matrix-valued x at 17-28 and
   // at 33-64 workers (TB/s rows / best other kernel; ring + ring fused K = 17 5.5/5.4, 21 5.9/4.6, 24 5.8/4.6,
   // 28 5.6/5.2, 33 5.7/3.7, 40 6.1/4.2, 48 6.2/4.7, 56 5.8/4.2, 64 5.7/4.8; matching fused 5.6-6.2/3.7-5.9; four slots
-  // 4.6-5.4/3.2-4.7; ring Mix2 with a matrix x K = 17 6.3/4.3, 24 6.4/4.3, 33 5.5/4.3, 40 5.5/5.2, 56 6.1/4.5; from 59
-  // workers its stages push the shared-memory carve-out to the maximum, the 28 KB of L1 left cannot hold the 30 KB
-  // of x that the rows' owners have in flight one tile ahead, and it falls to 4.8 against 5.0-5.4, so the
+  // 4.6-5.4/3.2-4.7; ring Mix2 with a matrix x K = 17 6.3/4.3, 24 6.4/4.3, 33 5.5/4.3, 40 5.5/5.2, 56 6.1/4.5; between 58
+  // and 60 workers it falls to 4.8 against 5.0-5.4 -- where its stages push the shared-memory carve-out to the
+  // maximum and 28 KB of L1 are left for the 30 KB of x in flight one tile ahead, the likely cause -- so the
   // tensor-core kernel keeps a matrix x there).  Not
   // with five and more slots in BOTH mixes from 25 workers, where the tensor-core kernels (Mix2, from 49 workers
   // also Mix1, as MMAs whatever the slot count) are ahead (K = 64, six slots: 4.1/4.8); not at 29-32 workers, where
