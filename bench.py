@@ -81,6 +81,7 @@ def parse_args():
                     help="instead of the round: the fused step across worker counts and mix kinds (4 GB per tensor)")
     ap.add_argument("--sweep-ks", default="", help="with --sweep: comma-separated worker counts (default: the full list)")
     ap.add_argument("--sweep-bytes", type=int, default=4_000_000_000, help="with --sweep: bytes per [K,P] tensor (smaller for an ncu capture)")
+    ap.add_argument("--sweep-standalone", action="store_true", help="with --sweep: time the stand-alone calls (fgd_mix ring / mean, fgd_consensus_distance) instead of the fused step")
     ap.add_argument("--kernels", action="store_true",
                     help="instead of the round: time every stand-alone C-ABI kernel of the config alone")
     ap.add_argument("--js", action="store_true",
@@ -501,7 +502,7 @@ def run_ours(args):
         if rank == 0:
             ks = tuple(int(k) for k in args.sweep_ks.split(",")) if args.sweep_ks else None
             print(json.dumps(sweep_table(torch, fgd, gen, dev, measured_peak(), tensor_bytes=args.sweep_bytes,
-                                         **({"Ks": ks} if ks else {}))), flush=True)
+                                         standalone=args.sweep_standalone, **({"Ks": ks} if ks else {}))), flush=True)
         return
     cfg = dict(CONFIGS[args.config])
     if args.cols:
@@ -649,7 +650,7 @@ def kernel_table(torch, fgd, drv, cfg, theta, local, mom, seed, dense_W, peak, r
 
 
 def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
-                Ks=(2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 20, 24, 28, 32, 40, 48, 56, 63, 64)):
+                Ks=(2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 20, 24, 28, 32, 40, 48, 56, 63, 64), standalone=False):
     """Fused outer step (in place, consensus sums on) across worker counts at a fixed tensor size:
     Mix2 = ring / hypercube (powers of two) / dense Sinkhorn with x one value per column, and the
     fully fused ring-ring and matching-matching (pairwise gossip for both mixes, App. A) rounds.  GB/s = algorithmic bytes (20 K P + 4 P, or 20 K P fused) / time."""
@@ -663,6 +664,26 @@ def sweep_table(torch, fgd, gen, dev, peak, tensor_bytes=4_000_000_000, reps=10,
         cd = torch.zeros(K, dtype=torch.float64, device=dev)
         ctx = fgd.Context(K, P, device=dev.index or 0)
         ring = fgd.MixDesc.ring(K)
+        if standalone:      # the stand-alone calls: 8 / 4 + 4/K / 4 algorithmic bytes per worker-parameter
+            out_t, xv, row = torch.empty_like(tp), torch.empty(P, dtype=torch.float32, device=dev), {}
+            mean = fgd.MixDesc.mean(K)
+            for name, f, nbytes in (("fgd_mix ring -> [K,P]", lambda: fgd.fgd_mix(ctx, ring, tp, out_t), 8 * K * P),
+                                    ("fgd_mix matching -> [K,P]", lambda: fgd.fgd_mix(ctx, fgd.MixDesc.random_matching(K, 0, 0, 1), tp, out_t), 8 * K * P),
+                                    ("fgd_mix mean -> [P]", lambda: fgd.fgd_mix(ctx, mean, tp, xv, out_is_vector=True), 4 * K * P + 4 * P),
+                                    ("fgd_consensus_distance", lambda: fgd.fgd_consensus_distance(ctx, tp, cd), 4 * K * P)):
+                for _ in range(3):
+                    f()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(reps):
+                    f()
+                b.record()
+                torch.cuda.synchronize()
+                row[name] = round(nbytes / (a.elapsed_time(b) / reps * 1e-3) / 1e9)
+            out["rows"][str(K)] = row
+            del tp, tl, v, x, out_t, xv
+            continue
         cases = {"ring": (ring, None), "dense": (fgd.MixDesc.dense(gen.sinkhorn_W(0, K)), None), "ring+ring fused": (ring, ring),
                  "matching+matching fused": (fgd.MixDesc.random_matching(K, 0, 0, 2), fgd.MixDesc.random_matching(K, 0, 0, 1))}
         if K & (K - 1) == 0 and K > 1:
